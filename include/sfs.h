@@ -1,0 +1,211 @@
+/*
+ * sfs.h — C ABI of libsfs: the per-step denoising hot path of SlowFast Sampling for masked-diffusion
+ * language models, for NVIDIA B200 (sm_100a).
+ *
+ * One denoising step (paper Section 3.1, Eqs. 2-4) is
+ *     logits = p_theta(prompt || partially masked response)        -> sfs_forward
+ *     r_hat_i, c_i = argmax / max softmax probability per row       -> sfs_row_stats
+ *     y^(k-1) = S(r_hat, y^(k), k)   with S the SlowFast rule        -> sfs_select
+ * and sfs_generate runs the whole loop of Algorithm 1 on the device.
+ *
+ * Conventions
+ *   * Every function returns an int32 status: SFS_OK (0) or a negative SFS_ERR_* code.  Nothing throws,
+ *     aborts or traps the device.  sfs_last_error() gives a human-readable message for the last failure
+ *     on the calling thread.
+ *   * Pointers whose name starts with d_ are DEVICE pointers owned by the caller; all others are HOST
+ *     pointers.  `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *     validate their arguments on the host, enqueue work on `stream` and return without synchronising,
+ *     unless stated otherwise.
+ *   * Tokens are int32 [B, S] row-major with S = P + L (prompt then response); `mask` is uint8 [B, S],
+ *     1 = position still masked.  A "row" is a flat token index b*S + pos.  Response positions are
+ *     0-based: i = pos - P.
+ *   * bf16 matrices are row-major with the contraction dimension contiguous: a weight of a layer that
+ *     maps in -> out is stored [out, in].
+ *   * Confidence comparisons are taken on the canonical fixed-point softmax denominator S_q (Q28, see
+ *     sfs_row_stats), never on a floating-point probability, so results do not depend on reduction order.
+ */
+#ifndef SFS_H_
+#define SFS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SFS_OK                 0
+#define SFS_ERR_INVALID_ARG   -1   /* null / misaligned pointer, size out of range, inconsistent shapes */
+#define SFS_ERR_UNSUPPORTED   -2   /* a shape this build has no kernel for */
+#define SFS_ERR_CUDA          -3   /* a CUDA runtime or driver call failed */
+#define SFS_ERR_OOM           -4   /* workspace allocation failed */
+#define SFS_ERR_STEP_LIMIT    -5   /* a sequence still had masked positions when its step budget ran out */
+#define SFS_ERR_TIMEOUT       -6   /* a bounded device-side wait gave up */
+#define SFS_ERR_MISSING_ROW   -7   /* the selection rule needed the statistics of a row that was not supplied */
+
+#define SFS_LOGITS_BF16 0
+#define SFS_LOGITS_F32  1
+
+#define SFS_PHASE_SLOW 0           /* exploratory stage (Section 3.3, stage 1) */
+#define SFS_PHASE_FAST 1           /* accelerated decoding stage (Section 3.3, stage 2) */
+
+#define SFS_CONF_QBITS 28          /* S_q = sum_v trunc(2^28 * exp(x_v - max x)) */
+#define SFS_MAX_W_HIST 8
+#define SFS_TRACE_INTS 8
+
+typedef struct sfs_model   sfs_model;     /* weights + shapes (borrowed device pointers) */
+typedef struct sfs_session sfs_session;   /* workspace for up to max_batch x max_seq tokens; one per host thread */
+
+/* Shape of the mask predictor (a pre-norm bidirectional transformer with RoPE, SwiGLU and RMSNorm). */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ff, vocab, mask_id;
+    float   rms_eps, rope_theta, logit_scale;
+} sfs_config;
+
+/* Device pointers to bf16 weights.  The per-layer members are HOST arrays of n_layers device pointers.
+ * Everything is borrowed: it must stay valid and unchanged for the life of the model. */
+typedef struct {
+    const void *tok_emb;      /* [vocab, d_model] */
+    const void *final_norm;   /* [d_model] */
+    const void *lm_head;      /* [vocab, d_model] */
+    const void *const *attn_norm;  /* [d_model] */
+    const void *const *wq, *const *wk, *const *wv, *const *wo;   /* [d_model, d_model] */
+    const void *const *mlp_norm;   /* [d_model] */
+    const void *const *w_gate, *const *w_up;   /* [d_ff, d_model] */
+    const void *const *w_down;                 /* [d_model, d_ff] */
+} sfs_weights;
+
+/* Hyper-parameters of the SlowFast rule (Section 3.3; defaults of Section 4.2 in comments). */
+typedef struct {
+    float   tau_min_conf;     /* 0.1   end-point threshold */
+    float   tau_high_conf;    /* 0.85  parallel-unmask threshold */
+    float   sigma2_stable;    /* 1.0   variance threshold of the stability check */
+    int32_t k_max;            /* 8     maximum exploratory steps per cycle */
+    int32_t w_hist;           /* 2     history window, 1..SFS_MAX_W_HIST */
+    int32_t k_slow;           /* 1     tokens unmasked per exploratory step */
+    int32_t k_fast;           /* 1     tokens unmasked by the fallback of an accelerated step */
+    int32_t max_steps;        /* N; 0 means N = gen_len */
+    int32_t min_high_count;   /* 1     fallback when fewer positions than this exceed tau_high_conf */
+} sfs_params;
+
+/* Per-sequence scheduler state, device-resident, plain data (Algorithm 1's k, s_cycle, e_cycle, H_W, step_count). */
+typedef struct {
+    int32_t phase;            /* SFS_PHASE_* of the NEXT step */
+    int32_t s_cycle;          /* start of the current cycle (response position) */
+    int32_t hi;               /* e_cycle + 1: end of the span, meaningful in the fast phase */
+    int32_t step_count;       /* exploratory steps taken in this cycle */
+    int32_t hist_len;
+    int32_t hist[SFS_MAX_W_HIST];   /* last e_cand values, oldest first */
+    int32_t k_remaining;      /* steps still permitted */
+    int32_t n_masked;
+    int32_t steps_done, n_slow, n_fast, n_cycles, n_fallback;
+    int32_t done;             /* 1 when no masked position is left (or the budget is spent) */
+    int32_t status;           /* SFS_OK or a SFS_ERR_* detected on the device */
+    int32_t reserved[12];
+} sfs_state;                  /* 32 int32 */
+
+/* ---- model and session ------------------------------------------------------------------------------ */
+
+/* Section 3.1 (the mask predictor p_theta).  Checks shapes (head_dim 64 or 128, n_heads*head_dim == d_model,
+ * d_model and d_ff multiples of 8, vocab a multiple of 8), copies the pointer tables and precomputes the
+ * RoPE table.  Allocates device memory; synchronises. */
+int32_t sfs_model_create(const sfs_config *cfg, const sfs_weights *weights, sfs_model **out);
+int32_t sfs_model_destroy(sfs_model *model);
+
+/* Allocates every buffer a forward / generate call over at most max_batch sequences of at most max_seq
+ * tokens needs (activations, logits [max_batch*max_seq, vocab] bf16, row statistics, scheduler scratch). */
+int32_t sfs_session_create(sfs_model *model, int32_t max_batch, int32_t max_seq, sfs_session **out);
+/* A session that can only run sfs_select (no model, hence no forward pass): allocates the selection
+ * scratch for max_batch x max_seq token positions and logits rows of `vocab` entries. */
+int32_t sfs_select_session_create(int32_t vocab, int32_t max_batch, int32_t max_seq, sfs_session **out);
+int32_t sfs_session_destroy(sfs_session *session);
+
+/* ---- the steps of one denoising iteration ----------------------------------------------------------- */
+
+/* Eq. 2: logits of the mask predictor for the listed rows.
+ *   d_tokens [B, S] int32 (masked positions must hold mask_id); d_rows [>= n_rows] flat token indices, or
+ *   NULL for all B*S rows in order; n_rows is read from the device scalar d_n_rows when it is not NULL
+ *   (then max_rows bounds it and sizes the launch), else it is max_rows.
+ *   d_logits [max_rows, vocab] row-major, bf16 or fp32 per logits_dtype; row r belongs to d_rows[r]. */
+int32_t sfs_forward(sfs_session *session, const int32_t *d_tokens, int32_t B, int32_t S,
+                    const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
+                    void *d_logits, int32_t logits_dtype, void *stream);
+
+/* Eq. 3 and the confidence equation of Section 3.1, per logits row:
+ *   argmax (lowest id among equal maxima), and S_q, the fixed-point softmax denominator
+ *       d = x_v - m;  r = fma(d, log2 e, 1.5*2^23);  n = r - 1.5*2^23;  f = fma(n, -ln 2, d);
+ *       P = 3 + f(C1 + f(C2 + f(C3 + f C4)));  e_v = ((bits(P) << 9) mod 2^32) >> (3 - n);  S_q = sum e_v
+ *   (fp32, each operation rounded once), so the confidence is c = 2^28 / S_q up to 1e-5 relative.
+ *   d_logits [n_rows, ld] (ld >= vocab elements between rows).  Outputs, each optional (NULL to skip):
+ *   d_argmax int32 [n_rows], d_sq uint64 [n_rows], d_conf float [n_rows] (= 2^28 / S_q, informational).
+ *   n_rows comes from d_n_rows when not NULL (bounded by max_rows).  Finite or -inf logits only. */
+int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
+                      const int32_t *d_n_rows, int32_t max_rows,
+                      int32_t *d_argmax, uint64_t *d_sq, float *d_conf, void *stream);
+
+/* Initial scheduler state for B sequences of gen_len masked positions (Algorithm 1, initialisation). */
+int32_t sfs_state_init(sfs_state *d_state, int32_t B, int32_t gen_len, const sfs_params *params, void *stream);
+
+/* Section 3.3 / Algorithm 1, one step of the transition rule S for B independent sequences:
+ * row statistics of the supplied logits, then per sequence the exploratory rule (top-k_slow unmasking,
+ * end point e_cand, history, variance test) or the accelerated rule (unmask every in-span position above
+ * tau_high_conf, else top-k_fast), the last-step rule (k == 1: unmask everything), and the phase / span
+ * bookkeeping.  Updates d_tokens, d_mask and d_state in place.
+ *   d_logits [n_rows, ld]; d_rows [n_rows] flat token indices b*S + pos the logits rows belong to; a
+ *   sequence's step needs the rows of its masked positions in [s_cycle, L) (slow), [s_cycle, hi) (fast) or
+ *   all of them (k_remaining == 1); extra rows are ignored, a missing one sets state.status =
+ *   SFS_ERR_MISSING_ROW and leaves the sequence untouched.
+ *   Outputs: d_sel_count [B], d_sel_pos / d_sel_tok [B, L] (response positions ascending, and their tokens);
+ *   optional d_next_rows [B*L] + d_next_n_rows [1]: the rows the following step will need, sequence-major;
+ *   optional d_trace [B, SFS_TRACE_INTS]: (phase, s_cycle, hi, e_cand, stable, n_sel, n_masked_after,
+ *   k_remaining_after) of this step. */
+int32_t sfs_select(sfs_session *session, const void *d_logits, int32_t logits_dtype, int64_t ld,
+                   const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
+                   int32_t *d_tokens, uint8_t *d_mask, int32_t B, int32_t S, int32_t P,
+                   sfs_state *d_state, const sfs_params *params,
+                   int32_t *d_sel_count, int32_t *d_sel_pos, int32_t *d_sel_tok,
+                   int32_t *d_next_rows, int32_t *d_next_n_rows, int32_t *d_trace, void *stream);
+
+/* ---- the whole loop ------------------------------------------------------------------------------------ */
+
+/* Algorithm 1 for B independent sequences with a common prompt length P and response length gen_len:
+ * loads prompt || [MASK]*gen_len into the session, runs denoising steps (forward, row statistics,
+ * selection, all on the device; finished sequences are skipped) until every sequence is done, and copies
+ * the tokens out.  d_prompt [B, P]; d_out_tokens [B, P + gen_len]; d_state_out [B] optional;
+ * d_trace [max_trace_steps, B, SFS_TRACE_INTS] optional.  Synchronises `stream` before returning and
+ * reports SFS_ERR_STEP_LIMIT / a device-detected status if any sequence did not finish cleanly.
+ * The three calls below split it so that a caller can run, time or checkpoint individual steps. */
+int32_t sfs_generate(sfs_session *session, const int32_t *d_prompt, int32_t B, int32_t P, int32_t gen_len,
+                     const sfs_params *params, int32_t *d_out_tokens, sfs_state *d_state_out,
+                     int32_t *d_trace, int32_t max_trace_steps, void *stream);
+
+int32_t sfs_generate_begin(sfs_session *session, const int32_t *d_prompt, int32_t B, int32_t P, int32_t gen_len,
+                           const sfs_params *params, void *stream);
+/* Enqueues up to n_steps denoising steps.  When d_logits_dump is not NULL, n_steps must be 1 and the bf16
+ * logits of that step ([max rows, vocab]), its row list and row count are copied there for inspection. */
+int32_t sfs_generate_steps(sfs_session *session, int32_t n_steps, int32_t *d_trace, int32_t max_trace_steps,
+                           void *d_logits_dump, int32_t *d_rows_dump, int32_t *d_n_rows_dump, void *stream);
+/* Synchronises; writes tokens / states; *n_active (host, optional) receives the number of unfinished sequences. */
+int32_t sfs_generate_end(sfs_session *session, int32_t *d_out_tokens, sfs_state *d_state_out,
+                         int32_t *n_active, int32_t *steps_enqueued, void *stream);
+
+/* ---- building blocks exposed for tests and measurements ------------------------------------------------- */
+
+/* C[M, N] = A[M, K] * B[N, K]^T, bf16 inputs, fp32 accumulation in tensor memory (tcgen05), output bf16
+ * (out_dtype 0) or fp32 (1), row-major with leading dimensions lda, ldb, ldc in elements.  The same kernel
+ * runs every projection of the forward pass.  K and the leading dimensions must be multiples of 8. */
+int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, void *d_C, int64_t ldc,
+                   int32_t M, int32_t N, int32_t K, int32_t out_dtype, float scale, void *stream);
+
+/* Bidirectional multi-head attention of one batch of sequences: d_qkv [B*S, 3*H*dh] bf16 (q | k | v per
+ * token, RoPE already applied to q and k), d_out [B*S, H*dh] bf16 = softmax(q k^T / sqrt(dh)) v within each
+ * sequence (no mask).  head_dim 64 or 128. */
+int32_t sfs_attention(sfs_session *session, const void *d_qkv, void *d_out, int32_t B, int32_t S, void *stream);
+
+const char *sfs_status_string(int32_t status);
+const char *sfs_last_error(void);
+int32_t     sfs_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SFS_H_ */

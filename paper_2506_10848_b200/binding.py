@@ -1,0 +1,130 @@
+"""ctypes binding of libsfs.so: same names as the C ABI (include/sfs.h), argument marshalling only.
+
+torch tensors are accepted wherever the ABI takes a device pointer (their data_ptr() is passed); every
+step of the path runs inside the library.  A missing or unloadable library raises: there is no fallback.
+"""
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int32, c_int64, c_uint64, c_void_p
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsfs.so")
+
+SFS_OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_OOM, ERR_STEP_LIMIT, ERR_TIMEOUT, ERR_MISSING_ROW = -1, -2, -3, -4, -5, -6, -7
+LOGITS_BF16, LOGITS_F32 = 0, 1
+PHASE_SLOW, PHASE_FAST = 0, 1
+CONF_QBITS = 28
+MAX_W_HIST = 8
+TRACE_INTS = 8
+
+
+class Config(Structure):
+    _fields_ = [(n, c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ff", "vocab", "mask_id")] + \
+               [(n, c_float) for n in ("rms_eps", "rope_theta", "logit_scale")]
+
+
+class Weights(Structure):
+    _fields_ = [("tok_emb", c_void_p), ("final_norm", c_void_p), ("lm_head", c_void_p)] + \
+               [(n, POINTER(c_void_p)) for n in ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down")]
+
+
+class Params(Structure):
+    _fields_ = [("tau_min_conf", c_float), ("tau_high_conf", c_float), ("sigma2_stable", c_float),
+                ("k_max", c_int32), ("w_hist", c_int32), ("k_slow", c_int32), ("k_fast", c_int32),
+                ("max_steps", c_int32), ("min_high_count", c_int32)]
+
+    @staticmethod
+    def default(**kw):
+        p = Params(0.1, 0.85, 1.0, 8, 2, 1, 1, 0, 1)
+        for k, v in kw.items():
+            setattr(p, k, v)
+        return p
+
+
+STATE_INTS = 32
+STATE_FIELDS = ["phase", "s_cycle", "hi", "step_count", "hist_len"] + [f"hist{i}" for i in range(MAX_W_HIST)] + \
+               ["k_remaining", "n_masked", "steps_done", "n_slow", "n_fast", "n_cycles", "n_fallback", "done", "status"]
+
+_lib = None
+
+
+class SfsError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"libsfs status {status}: {message}")
+        self.status = status
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with `python -m paper_2506_10848_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        L.sfs_last_error.restype = c_char_p
+        L.sfs_status_string.restype = c_char_p
+        L.sfs_status_string.argtypes = [c_int32]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    """torch tensor / int / None -> c_void_p."""
+    if t is None:
+        return c_void_p(0)
+    if isinstance(t, int):
+        return c_void_p(t)
+    return c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return c_void_p(torch.cuda.current_stream().cuda_stream)
+    if isinstance(stream, int):
+        return c_void_p(stream)
+    return c_void_p(stream.cuda_stream)
+
+
+def _check(rc):
+    if rc != SFS_OK:
+        raise SfsError(rc, lib().sfs_last_error().decode())
+
+
+def sfs_last_error():
+    return lib().sfs_last_error().decode()
+
+
+def sfs_status_string(status):
+    return lib().sfs_status_string(status).decode()
+
+
+def sfs_version():
+    return lib().sfs_version()
+
+
+def sfs_row_stats(logits, logits_dtype, vocab, ld, n_rows_dev, max_rows, argmax=None, sq=None, conf=None, stream=None):
+    _check(lib().sfs_row_stats(_ptr(logits), c_int32(logits_dtype), c_int32(vocab), c_int64(ld), _ptr(n_rows_dev),
+                               c_int32(max_rows), _ptr(argmax), _ptr(sq), _ptr(conf), _stream(stream)))
+
+
+def sfs_state_init(state, B, gen_len, params, stream=None):
+    _check(lib().sfs_state_init(_ptr(state), c_int32(B), c_int32(gen_len), byref(params), _stream(stream)))
+
+
+def sfs_select_session_create(vocab, max_batch, max_seq):
+    h = c_void_p()
+    _check(lib().sfs_select_session_create(c_int32(vocab), c_int32(max_batch), c_int32(max_seq), byref(h)))
+    return h
+
+
+def sfs_session_destroy(session):
+    _check(lib().sfs_session_destroy(session))
+
+
+def sfs_select(session, logits, logits_dtype, ld, rows, n_rows_dev, max_rows, tokens, mask, B, S, P, state, params,
+               sel_count=None, sel_pos=None, sel_tok=None, next_rows=None, next_n_rows=None, trace=None, stream=None):
+    _check(lib().sfs_select(session, _ptr(logits), c_int32(logits_dtype), c_int64(ld), _ptr(rows), _ptr(n_rows_dev),
+                            c_int32(max_rows), _ptr(tokens), _ptr(mask), c_int32(B), c_int32(S), c_int32(P),
+                            _ptr(state), byref(params), _ptr(sel_count), _ptr(sel_pos), _ptr(sel_tok),
+                            _ptr(next_rows), _ptr(next_n_rows), _ptr(trace), _stream(stream)))

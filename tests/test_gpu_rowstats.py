@@ -1,0 +1,85 @@
+"""GPU parity: row statistics (greedy token, canonical softmax denominator) against the oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rowstats as RS
+from paper_2506_10848_b200 import binding as sfs
+from paper_2506_10848_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def gpu_stats(logits, vocab, ld, dtype, n_rows_dev=None, max_rows=None):
+    R = logits.shape[0] if max_rows is None else max_rows
+    arg = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    sq = torch.full((R,), -7, dtype=torch.int64, device=DEV)
+    conf = torch.full((R,), -7.0, dtype=torch.float32, device=DEV)
+    sfs.sfs_row_stats(logits, dtype, vocab, ld, n_rows_dev, R, argmax=arg, sq=sq, conf=conf)
+    torch.cuda.synchronize()
+    return arg.cpu().numpy(), sq.cpu().numpy().view(np.uint64), conf.cpu().numpy()
+
+
+@pytest.mark.parametrize("R,V", [(1, 8), (3, 64), (5, 2048), (7, 4096), (4, 4104), (6, 16384), (3, 32768 + 64),
+                                 (5, 65536 + 8), (9, 126464), (2, 131072)])
+def test_bf16_fast_path_matches_oracle(R, V):
+    x = W.planted_logits(R, V, seed=100 + R, device="cpu")
+    if R > 2:
+        x[1, :] = x[1, 0]                                   # a fully tied row
+        x[2, V // 2] = x[2].max()                           # a duplicated maximum
+    ref = RS.row_stats(W.bf16_bits(x))
+    arg, sq, conf = gpu_stats(x.to(DEV), V, V, sfs.LOGITS_BF16)
+    assert np.array_equal(arg, ref["argmax"])
+    assert np.array_equal(sq, ref["sq"])
+    assert np.allclose(conf, ref["conf_exact"], rtol=2e-5, atol=V * 2.0 ** -28)
+
+
+@pytest.mark.parametrize("V,ld", [(1, 1), (7, 7), (1000, 1003), (4095, 4096), (126463, 126464)])
+def test_generic_paths_match_oracle(V, ld):
+    R = 5
+    g = torch.Generator().manual_seed(V)
+    full = (torch.randn((R, ld), generator=g) * 3).to(torch.float32)
+    full[0, V // 2] += 9.0
+    ref32 = RS.row_stats(np.ascontiguousarray(full[:, :V].numpy()))
+    arg, sq, _ = gpu_stats(full.to(DEV), V, ld, sfs.LOGITS_F32)
+    assert np.array_equal(arg, ref32["argmax"]) and np.array_equal(sq, ref32["sq"])
+    fb = full.to(torch.bfloat16)
+    refb = RS.row_stats(np.ascontiguousarray(W.bf16_bits(fb)[:, :V]))
+    arg, sq, _ = gpu_stats(fb.to(DEV), V, ld, sfs.LOGITS_BF16)          # odd V / ld: the generic bf16 kernel
+    assert np.array_equal(arg, refb["argmax"]) and np.array_equal(sq, refb["sq"])
+
+
+def test_special_values_and_device_row_count():
+    V = 4096
+    x = torch.zeros((6, V), dtype=torch.float32)
+    x[0] = -float("inf"); x[0, 17] = 2.0; x[0, 900] = 1.0              # -inf entries contribute nothing
+    x[1, 5] = 3e38; x[1, 6] = -3e38                                      # huge spread
+    x[2] = -1e4; x[2, V - 1] = -9990.0                                   # maximum in the last column
+    x[3, 0] = 0.0; x[3, 1] = -0.0                                        # +0 == -0: lowest id wins
+    x[4] = torch.linspace(-30, 30, V)
+    x[5] = -float("inf")                                                 # nothing finite at all
+    xb = x.to(torch.bfloat16)
+    ref = RS.row_stats(W.bf16_bits(xb))
+    n = torch.tensor([5], dtype=torch.int32, device=DEV)                 # device-side row count: row 5 is skipped
+    arg, sq, _ = gpu_stats(xb.to(DEV), V, V, sfs.LOGITS_BF16, n_rows_dev=n, max_rows=6)
+    assert np.array_equal(arg[:5], ref["argmax"][:5]) and np.array_equal(sq[:5], ref["sq"][:5])
+    assert arg[5] == -7                                                  # untouched
+    arg, sq, _ = gpu_stats(xb.to(DEV), V, V, sfs.LOGITS_BF16)
+    assert np.array_equal(arg, ref["argmax"]) and np.array_equal(sq, ref["sq"])
+    ref32 = RS.row_stats(np.ascontiguousarray(x.numpy()))
+    arg, sq, _ = gpu_stats(x.to(DEV), V, V, sfs.LOGITS_F32)
+    assert np.array_equal(arg, ref32["argmax"]) and np.array_equal(sq, ref32["sq"])
+
+
+def test_epilogue_microbenchmark_shape_full_size():
+    """The sampling-epilogue workload at full size: bf16 [256, 126464], planted winners."""
+    x = W.planted_logits(256, 126464, seed=1, device="cpu")
+    ref = RS.row_stats(W.bf16_bits(x))
+    arg, sq, conf = gpu_stats(x.to(DEV), 126464, 126464, sfs.LOGITS_BF16)
+    assert np.array_equal(arg, ref["argmax"])
+    assert np.array_equal(sq, ref["sq"])
+    assert np.allclose(conf, ref["conf_exact"], rtol=2e-5, atol=126464 * 2.0 ** -28)
+    # run-to-run determinism
+    arg2, sq2, _ = gpu_stats(x.to(DEV), 126464, 126464, sfs.LOGITS_BF16)
+    assert np.array_equal(sq, sq2) and np.array_equal(arg, arg2)

@@ -1,0 +1,182 @@
+"""GPU parity: one step of the SlowFast rule (row statistics + selection) against the oracle's step machine,
+bit for bit, driven with seeded synthetic logits whose confidences fire every branch."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rowstats as RS
+from oracle.scheduler import FAST, SLOW, SlowFastState, rows_needed, slowfast_step
+from paper_2506_10848_b200 import binding as sfs
+from paper_2506_10848_b200 import workloads as W
+
+from helpers import oracle_state_as_ints, params_pair, state_to_dict, write_state
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def synthetic_step_logits(n_rows, V, gen, dtype):
+    """Rows with a planted winner whose margin makes confidences spread over (0, 1)."""
+    x = torch.randn((n_rows, V), generator=gen) * 1.5
+    col = torch.randint(0, V, (n_rows,), generator=gen)
+    margin = torch.rand((n_rows,), generator=gen) * 14.0
+    x[torch.arange(n_rows), col] = x.max(dim=1).values + margin
+    return x.to(dtype)
+
+
+def run_lockstep(B, P, L, V, pkw, seed, dtype=torch.bfloat16, supply_all_rows=False):
+    po, pg = params_pair(**pkw)
+    S = P + L
+    gen = torch.Generator().manual_seed(seed)
+    session = sfs.sfs_select_session_create(V, B, S)
+    try:
+        tokens = torch.full((B, S), V - 1, dtype=torch.int32, device=DEV)
+        mask = torch.zeros((B, S), dtype=torch.uint8, device=DEV); mask[:, P:] = 1
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+        sfs.sfs_state_init(state, B, L, pg)
+        sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+        sel_pos = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+        sel_tok = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+        next_rows = torch.zeros(B * L, dtype=torch.int32, device=DEV)
+        next_n = torch.zeros(1, dtype=torch.int32, device=DEV)
+        trace = torch.zeros((B, sfs.TRACE_INTS), dtype=torch.int32, device=DEV)
+        ost = [SlowFastState.fresh(L, po) for _ in range(B)]
+        oy = [[None] * L for _ in range(B)]
+        steps = 0
+        while not all(s.done for s in ost):
+            need = [(b, i) for b in range(B) for i in rows_needed(ost[b])]
+            if steps > 0:                                   # the library's own row list for this step
+                n = int(next_n.item())
+                assert next_rows[:n].tolist() == [b * S + P + i for (b, i) in need]
+            rows_list = need
+            if supply_all_rows:                             # extra rows must be ignored
+                rows_list = [(b, i) for b in range(B) for i in range(L) if ost[b].masked[i] and not ost[b].done]
+            n_rows = len(rows_list)
+            logits = synthetic_step_logits(n_rows, V, gen, dtype)
+            rows = torch.tensor([b * S + P + i for (b, i) in rows_list], dtype=torch.int32, device=DEV)
+            n_dev = torch.tensor([n_rows], dtype=torch.int32, device=DEV)
+            dl = logits.to(DEV)
+            sfs.sfs_select(session, dl, sfs.LOGITS_BF16 if dtype == torch.bfloat16 else sfs.LOGITS_F32, V, rows, n_dev,
+                           n_rows, tokens, mask, B, S, P, state, pg, sel_count, sel_pos, sel_tok, next_rows, next_n, trace)
+            torch.cuda.synchronize()
+            st = RS.row_stats(W.bf16_bits(logits) if dtype == torch.bfloat16 else logits.numpy())
+            for b in range(B):
+                if ost[b].done:
+                    assert int(sel_count[b]) == 0
+                    continue
+                idx = {i: j for j, (bb, i) in enumerate(rows_list) if bb == b}
+                a = {i: int(st["argmax"][j]) for i, j in idx.items()}
+                sq = {i: int(st["sq"][j]) for i, j in idx.items()}
+                rec = slowfast_step(ost[b], a, sq, po)
+                for i, t in zip(rec.positions, rec.tokens):
+                    oy[b][i] = t
+                n = int(sel_count[b])
+                assert sel_pos[b, :n].tolist() == rec.positions
+                assert sel_tok[b, :n].tolist() == rec.tokens
+                tr = trace[b].tolist()
+                assert tr[:6] == [rec.phase, rec.s, rec.hi, rec.e_cand, rec.stable, len(rec.positions)]
+                got = state_to_dict(state[b])
+                want = oracle_state_as_ints(ost[b], po.w_hist)
+                if ost[b].done:                                   # phase / span of a finished sequence carry no meaning
+                    want = {k: want[k] for k in ("n_masked", "done", "k_remaining")}
+                for k_, v_ in want.items():
+                    assert got[k_] == v_, (k_, got, want)
+                assert got["status"] == 0
+            steps += 1
+            assert steps <= (po.max_steps or L) + 1
+        tk = tokens.cpu()
+        mk = mask.cpu()
+        for b in range(B):
+            assert tk[b, P:].tolist() == oy[b]
+            assert int(mk[b].sum()) == 0
+        return steps
+    finally:
+        sfs.sfs_session_destroy(session)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_lockstep_default_params(seed):
+    steps = run_lockstep(B=3, P=5, L=48, V=512, pkw={}, seed=seed)
+    assert steps < 48                                       # parallel unmasking happened
+
+
+@pytest.mark.parametrize("seed,pkw", [
+    (10, dict(k_max=3, w_hist=3, sigma2_stable=30.0, k_slow=2, k_fast=3)),
+    (11, dict(k_max=1, w_hist=1, k_slow=4, min_high_count=3)),
+    (12, dict(max_steps=9, k_slow=1)),                       # the step budget runs out: forced last step
+    (13, dict(tau_min_conf=-1.0, tau_high_conf=2.0, sigma2_stable=float("inf"), k_max=1, w_hist=1)),
+    (14, dict(w_hist=8, k_max=12, sigma2_stable=400.0)),
+])
+def test_lockstep_other_params(seed, pkw):
+    run_lockstep(B=2, P=3, L=40, V=256, pkw=pkw, seed=seed)
+
+
+def test_lockstep_fp32_logits_extra_rows_and_ragged_sizes():
+    run_lockstep(B=1, P=0, L=1, V=8, pkw={}, seed=20, dtype=torch.float32)
+    run_lockstep(B=4, P=7, L=33, V=1000, pkw={}, seed=21, dtype=torch.float32, supply_all_rows=True)
+    run_lockstep(B=2, P=1, L=300, V=512, pkw=dict(k_slow=3), seed=22, supply_all_rows=True)
+
+
+def test_missing_row_is_reported_not_guessed():
+    po, pg = params_pair()
+    B, P, L, V = 1, 2, 8, 64
+    S = P + L
+    session = sfs.sfs_select_session_create(V, B, S)
+    try:
+        tokens = torch.full((B, S), V - 1, dtype=torch.int32, device=DEV)
+        mask = torch.zeros((B, S), dtype=torch.uint8, device=DEV); mask[:, P:] = 1
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+        sfs.sfs_state_init(state, B, L, pg)
+        logits = torch.randn((L - 1, V)).to(torch.bfloat16).to(DEV)      # the row of position L-1 is withheld
+        rows = torch.arange(P, P + L - 1, dtype=torch.int32, device=DEV)
+        sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+        sfs.sfs_select(session, logits, sfs.LOGITS_BF16, V, rows, None, L - 1, tokens, mask, B, S, P, state, pg, sel_count)
+        torch.cuda.synchronize()
+        assert state_to_dict(state[0])["status"] == sfs.ERR_MISSING_ROW
+        assert int(sel_count[0]) == 0 and int(mask.sum()) == L
+    finally:
+        sfs.sfs_session_destroy(session)
+
+
+def test_epilogue_microbenchmark_one_slow_one_fast_step():
+    """bf16 logits [256, 126464] with planted winners; one exploratory and one accelerated step from a given
+    span [lo, hi), compared with the oracle."""
+    V, L, P, B = 126464, 256, 0, 1
+    po, pg = params_pair()
+    x = W.planted_logits(L, V, seed=1, device="cpu")
+    st = RS.row_stats(W.bf16_bits(x))
+    frac = [float(np.mean(RS.exceeds(st["sq"], t))) for t in (0.1, 0.85, 0.9)]
+    print("fraction of rows above 0.1 / 0.85 / 0.9:", frac)
+    lo, hi = W.span(L, seed=1)
+    dl = x.to(DEV)
+    session = sfs.sfs_select_session_create(V, B, L)
+    try:
+        for phase in (SLOW, FAST):
+            tokens = torch.full((B, L), V - 1, dtype=torch.int32, device=DEV)
+            mask = torch.ones((B, L), dtype=torch.uint8, device=DEV); mask[:, :lo] = 0
+            state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+            sfs.sfs_state_init(state, B, L, pg)
+            write_state(state, 0, phase=phase, s_cycle=lo, hi=hi if phase == FAST else 0, n_masked=L - lo,
+                        k_remaining=L - lo, hist_len=1 if phase == SLOW else 0, hist0=L - 1, step_count=1 if phase == SLOW else 0)
+            ost = SlowFastState(L=L, k=L - lo, phase=phase, s_cycle=lo, hi=hi if phase == FAST else 0,
+                                step_count=1 if phase == SLOW else 0, H=[L - 1] if phase == SLOW else [],
+                                masked=[i >= lo for i in range(L)])
+            need = rows_needed(ost)
+            rows = torch.tensor(need, dtype=torch.int32, device=DEV)
+            sub = dl[need].contiguous()
+            sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+            sel_pos = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+            sel_tok = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+            sfs.sfs_select(session, sub, sfs.LOGITS_BF16, V, rows, None, len(need), tokens, mask, B, L, P, state, pg,
+                           sel_count, sel_pos, sel_tok)
+            torch.cuda.synchronize()
+            rec = slowfast_step(ost, {i: int(st["argmax"][i]) for i in need}, {i: int(st["sq"][i]) for i in need}, po)
+            n = int(sel_count[0])
+            assert sel_pos[0, :n].tolist() == rec.positions and sel_tok[0, :n].tolist() == rec.tokens
+            got = state_to_dict(state[0])
+            for k_, v_ in oracle_state_as_ints(ost, po.w_hist).items():
+                assert got[k_] == v_, (k_, got)
+            if phase == FAST:
+                assert n > 1                               # several in-span rows exceed tau_high: parallel unmasking
+    finally:
+        sfs.sfs_session_destroy(session)
