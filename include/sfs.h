@@ -100,8 +100,8 @@ typedef struct {
     int32_t steps_done, n_slow, n_fast, n_cycles, n_fallback;
     int32_t done;             /* 1 when no masked position is left (or the budget is spent) */
     int32_t status;           /* SFS_OK or a SFS_ERR_* detected on the device */
-    int32_t reserved[12];
-} sfs_state;                  /* 32 int32 */
+    int32_t reserved[10];
+} sfs_state;                  /* 32 int32 = 128 bytes */
 
 /* ---- model and session ------------------------------------------------------------------------------ */
 

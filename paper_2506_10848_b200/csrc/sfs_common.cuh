@@ -9,6 +9,8 @@
 
 #include "../../include/sfs.h"
 
+static_assert(sizeof(sfs_state) == 128, "sfs_state is 32 int32");
+
 namespace sfs {
 
 // ---- host-side error reporting ---------------------------------------------------------------------
