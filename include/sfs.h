@@ -201,6 +201,10 @@ int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, v
  * sequence (no mask).  head_dim 64 or 128. */
 int32_t sfs_attention(sfs_session *session, const void *d_qkv, void *d_out, int32_t B, int32_t S, void *stream);
 
+/* Synchronises `stream` and returns (then clears) the sticky device status word: SFS_OK, or SFS_ERR_TIMEOUT
+ * if a kernel's bounded wait gave up since the last check. */
+int32_t sfs_check_device_status(void *stream);
+
 const char *sfs_status_string(int32_t status);
 const char *sfs_last_error(void);
 int32_t     sfs_version(void);

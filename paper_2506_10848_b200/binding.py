@@ -128,3 +128,14 @@ def sfs_select(session, logits, logits_dtype, ld, rows, n_rows_dev, max_rows, to
                             c_int32(max_rows), _ptr(tokens), _ptr(mask), c_int32(B), c_int32(S), c_int32(P),
                             _ptr(state), byref(params), _ptr(sel_count), _ptr(sel_pos), _ptr(sel_tok),
                             _ptr(next_rows), _ptr(next_n_rows), _ptr(trace), _stream(stream)))
+
+
+def sfs_linear(A, lda, Bm, ldb, C, ldc, M, N, K, out_dtype=0, scale=1.0, stream=None):
+    _check(lib().sfs_linear(_ptr(A), c_int64(lda), _ptr(Bm), c_int64(ldb), _ptr(C), c_int64(ldc), c_int32(M), c_int32(N),
+                            c_int32(K), c_int32(out_dtype), c_float(scale), _stream(stream)))
+
+
+def sfs_check_device_status(stream=None):
+    rc = lib().sfs_check_device_status(_stream(stream))
+    if rc != SFS_OK:
+        raise SfsError(rc, lib().sfs_last_error().decode())

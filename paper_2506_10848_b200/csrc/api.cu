@@ -2,6 +2,7 @@
 // the order in which the kernels of one denoising step are enqueued.
 #include "sfs_common.cuh"
 #include "model.cuh"
+#include "gemm.cuh"
 
 #include <new>
 #include <string.h>
@@ -28,6 +29,17 @@ static int32_t check_params(const sfs_params *p)
     SFS_REQUIRE(p->sigma2_stable == p->sigma2_stable && p->tau_min_conf == p->tau_min_conf && p->tau_high_conf == p->tau_high_conf,
                 SFS_ERR_INVALID_ARG, "NaN threshold");
     return SFS_OK;
+}
+
+// one sticky device status word per process (set by kernels whose bounded waits give up)
+int32_t *device_status_word()
+{
+    static int32_t *w = nullptr;
+    if (!w) {
+        if (cudaMalloc(&w, 256) != cudaSuccess) { w = nullptr; return nullptr; }
+        cudaMemset(w, 0, 256);
+    }
+    return w;
 }
 
 }  // namespace sfs
@@ -162,6 +174,39 @@ int32_t sfs_select_session_create(int32_t vocab, int32_t max_batch, int32_t max_
     SFS_CUDA(cudaDeviceSynchronize());
     *out = s;
     return SFS_OK;
+}
+
+}  // extern "C"
+
+extern "C" {
+
+int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, void *d_C, int64_t ldc,
+                   int32_t M, int32_t N, int32_t K, int32_t out_dtype, float scale, void *stream)
+{
+    SFS_REQUIRE(d_A && d_B && d_C, SFS_ERR_INVALID_ARG, "linear: NULL pointer");
+    SFS_REQUIRE(M >= 1 && N >= 1 && K >= 1, SFS_ERR_INVALID_ARG, "linear: M, N, K must be positive");
+    SFS_REQUIRE(out_dtype == 0 || out_dtype == 1, SFS_ERR_INVALID_ARG, "linear: out_dtype %d", out_dtype);
+    int32_t *err = device_status_word();
+    SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
+    GemmPlan plan;
+    const void *bs[1] = {d_B};
+    int32_t rc = gemm_plan_create(&plan, d_A, lda, M, K, bs, 1, N, ldb, GEMM_STORE, d_C, ldc, out_dtype, scale, nullptr, 0, 0, 0);
+    if (rc != SFS_OK) return rc;
+    return gemm_launch(plan, nullptr, err, (cudaStream_t)stream);
+}
+
+int32_t sfs_check_device_status(void *stream)
+{
+    int32_t *err = device_status_word();
+    SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
+    SFS_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    int32_t h = 0;
+    SFS_CUDA(cudaMemcpy(&h, err, 4, cudaMemcpyDeviceToHost));
+    if (h != 0) {
+        cudaMemset(err, 0, 4);
+        set_error("a kernel reported device status %d (%s)", h, sfs_status_string(h));
+    }
+    return h;
 }
 
 }  // extern "C"

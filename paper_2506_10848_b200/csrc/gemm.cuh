@@ -1,0 +1,40 @@
+// Internal interface of the tcgen05 GEMM (C = A * B^T, bf16 in, fp32 accumulate).
+#pragma once
+#include "sfs_common.cuh"
+#include <cuda.h>
+#include <string.h>
+
+namespace sfs {
+
+enum GemmMode {
+    GEMM_STORE = 0,          // C = scale * acc   (bf16 or fp32); optionally the trailing columns go transposed to `vt`
+    GEMM_RESIDUAL_F32 = 1,   // C (fp32) += acc
+    GEMM_SWIGLU = 2,         // C (bf16) = silu(acc_gate) * acc_up, gate and up rows loaded side by side into one tile
+};
+
+struct GemmArgs {
+    int M, N, K;
+    const int32_t *d_m;      // optional device-side row count (<= M)
+    int mode, out_f32;
+    float scale;
+    void *C; long long ldc;
+    __nv_bfloat16 *vt; long long ldvt; int vt_col0;
+    int tiles_per_map;
+    int32_t *err;            // device status word, set to SFS_ERR_TIMEOUT if a bounded wait gives up
+};
+
+struct GemmPlan {
+    CUtensorMap tmA, tmB[3];
+    GemmArgs args;
+    int bn, n_maps, n_per_map;
+};
+
+// Bs: n_maps weight matrices [n_per_map, K] (ldb elements between rows) whose outputs are concatenated along
+// the columns of C (QKV), or gate / up for GEMM_SWIGLU (then C has n_per_map columns).
+int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int32_t K,
+                         const void *const *Bs, int32_t n_maps, int32_t n_per_map, int64_t ldb,
+                         int32_t mode, void *C, int64_t ldc, int32_t out_f32, float scale,
+                         __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, int32_t force_bn);
+int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, int32_t *err, cudaStream_t stream);
+
+}  // namespace sfs
