@@ -196,10 +196,14 @@ int32_t sfs_generate_end(sfs_session *session, int32_t *d_out_tokens, sfs_state 
 int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, void *d_C, int64_t ldc,
                    int32_t M, int32_t N, int32_t K, int32_t out_dtype, float scale, void *stream);
 
-/* Bidirectional multi-head attention of one batch of sequences: d_qkv [B*S, 3*H*dh] bf16 (q | k | v per
- * token, RoPE already applied to q and k), d_out [B*S, H*dh] bf16 = softmax(q k^T / sqrt(dh)) v within each
- * sequence (no mask).  head_dim 64 or 128. */
-int32_t sfs_attention(sfs_session *session, const void *d_qkv, void *d_out, int32_t B, int32_t S, void *stream);
+/* Bidirectional multi-head attention (the "a = softmax(q k^T / sqrt(dh)) v" of the mask predictor) over B
+ * sequences of S tokens, no mask, in the layout the forward pass uses internally:
+ *   d_qk  [B*S, 2*H*dh] bf16, per token q (H*dh values, RoPE applied) then k (H*dh values, RoPE applied);
+ *   d_vt  [H*dh, B*S]   bf16, V transposed (feature-major);
+ *   d_out [B*S, H*dh]   bf16.
+ * head_dim 64 or 128; S a multiple of 8. */
+int32_t sfs_attention(const void *d_qk, const void *d_vt, void *d_out, int32_t B, int32_t S,
+                      int32_t n_heads, int32_t head_dim, void *stream);
 
 /* Synchronises `stream` and returns (then clears) the sticky device status word: SFS_OK, or SFS_ERR_TIMEOUT
  * if a kernel's bounded wait gave up since the last check. */

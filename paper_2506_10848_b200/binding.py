@@ -139,3 +139,66 @@ def sfs_check_device_status(stream=None):
     rc = lib().sfs_check_device_status(_stream(stream))
     if rc != SFS_OK:
         raise SfsError(rc, lib().sfs_last_error().decode())
+
+
+def sfs_attention(qk, vt, out, B, S, n_heads, head_dim, stream=None):
+    _check(lib().sfs_attention(_ptr(qk), _ptr(vt), _ptr(out), c_int32(B), c_int32(S), c_int32(n_heads), c_int32(head_dim),
+                               _stream(stream)))
+
+
+class Model:
+    """Owns the sfs_model handle and keeps the weight tensors (borrowed by the library) alive."""
+
+    def __init__(self, shape, weights):
+        """shape: an object with the sfs_config field names; weights: dict of CUDA bf16 tensors as produced by
+        workloads.model_weights(..., device='cuda')."""
+        self.cfg = Config(*(int(getattr(shape, n)) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ff", "vocab", "mask_id")),
+                          *(float(getattr(shape, n)) for n in ("rms_eps", "rope_theta", "logit_scale")))
+        self.weights = weights
+        nl = self.cfg.n_layers
+        self._tables = {}
+        w = Weights()
+        w.tok_emb, w.final_norm, w.lm_head = (weights[k].data_ptr() for k in ("tok_emb", "final_norm", "lm_head"))
+        for name in ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "w_gate", "w_up", "w_down"):
+            arr = (c_void_p * nl)(*[weights["layers"][l][name].data_ptr() for l in range(nl)])
+            self._tables[name] = arr
+            setattr(w, name, ctypes.cast(arr, POINTER(c_void_p)))
+        self.handle = c_void_p()
+        _check(lib().sfs_model_create(byref(self.cfg), byref(w), byref(self.handle)))
+
+    def close(self):
+        if self.handle:
+            lib().sfs_model_destroy(self.handle)
+            self.handle = c_void_p()
+
+
+def sfs_session_create(model, max_batch, max_seq):
+    h = c_void_p()
+    _check(lib().sfs_session_create(model.handle if isinstance(model, Model) else model, c_int32(max_batch), c_int32(max_seq), byref(h)))
+    return h
+
+
+def sfs_forward(session, tokens, B, S, rows, n_rows_dev, max_rows, logits, logits_dtype, stream=None):
+    _check(lib().sfs_forward(session, _ptr(tokens), c_int32(B), c_int32(S), _ptr(rows), _ptr(n_rows_dev), c_int32(max_rows),
+                             _ptr(logits), c_int32(logits_dtype), _stream(stream)))
+
+
+def sfs_generate(session, prompt, B, P, gen_len, params, out_tokens, state_out=None, trace=None, max_trace_steps=0, stream=None):
+    _check(lib().sfs_generate(session, _ptr(prompt), c_int32(B), c_int32(P), c_int32(gen_len), byref(params), _ptr(out_tokens),
+                              _ptr(state_out), _ptr(trace), c_int32(max_trace_steps), _stream(stream)))
+
+
+def sfs_generate_begin(session, prompt, B, P, gen_len, params, stream=None):
+    _check(lib().sfs_generate_begin(session, _ptr(prompt), c_int32(B), c_int32(P), c_int32(gen_len), byref(params), _stream(stream)))
+
+
+def sfs_generate_steps(session, n_steps, trace=None, max_trace_steps=0, logits_dump=None, rows_dump=None, n_rows_dump=None, stream=None):
+    _check(lib().sfs_generate_steps(session, c_int32(n_steps), _ptr(trace), c_int32(max_trace_steps), _ptr(logits_dump),
+                                    _ptr(rows_dump), _ptr(n_rows_dump), _stream(stream)))
+
+
+def sfs_generate_end(session, out_tokens=None, state_out=None, stream=None):
+    """Returns (n_active, steps_enqueued)."""
+    na, ns = c_int32(0), c_int32(0)
+    _check(lib().sfs_generate_end(session, _ptr(out_tokens), _ptr(state_out), byref(na), byref(ns), _stream(stream)))
+    return na.value, ns.value

@@ -3,6 +3,8 @@
 #include "sfs_common.cuh"
 #include "model.cuh"
 #include "gemm.cuh"
+#include "attention.cuh"
+#include "elementwise.cuh"
 
 #include <new>
 #include <string.h>
@@ -42,6 +44,110 @@ int32_t *device_status_word()
     return w;
 }
 
+template <typename T>
+static int32_t dev_alloc(sfs_session *s, T **out, size_t count, bool zero)
+{
+    void *p = nullptr;
+    const size_t bytes = count * sizeof(T) > 0 ? count * sizeof(T) : 16;
+    SFS_CUDA(cudaMalloc(&p, bytes));
+    s->owned.push_back(p);
+    if (zero) SFS_CUDA(cudaMemset(p, 0, bytes));
+    *out = reinterpret_cast<T *>(p);
+    return SFS_OK;
+}
+
+static int32_t session_alloc_select(sfs_session *s)
+{
+    const size_t n = (size_t)s->max_batch * s->max_seq;
+    int32_t rc;
+    if ((rc = dev_alloc(s, &s->pos_sq, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->pos_arg, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->seq_rows, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->seq_row_count, (size_t)s->max_batch, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->ticket, 4, true)) != SFS_OK) return rc;
+    return SFS_OK;
+}
+
+// (re)build the GEMM / attention plans of a model session for B sequences of S tokens
+static int32_t session_plan(sfs_session *s, int32_t B, int32_t S)
+{
+    if (s->plan_B == B && s->plan_S == S) return SFS_OK;
+    const sfs_model *m = s->model;
+    const sfs_config &c = m->cfg;
+    const int T = B * S, d = c.d_model, ff = c.d_ff;
+    SFS_REQUIRE((S % 8) == 0, SFS_ERR_UNSUPPORTED, "sequence length %d must be a multiple of 8", S);
+    s->layer_plans.resize(c.n_layers);
+    int32_t rc;
+    for (int l = 0; l < c.n_layers; ++l) {
+        LayerPlans &lp = s->layer_plans[l];
+        const void *qkv[3] = {m->wq[l], m->wk[l], m->wv[l]};
+        // q | k go row-major into qk [T, 2d]; the v columns (>= 2d) go transposed into vt [d, T]
+        rc = gemm_plan_create(&lp.qkv, s->h, d, T, d, qkv, 3, d, d, GEMM_STORE, s->qk, 2 * d, 0, 1.0f, s->vt, T, 2 * d, 0);
+        if (rc != SFS_OK) return rc;
+        const void *wo[1] = {m->wo[l]};
+        rc = gemm_plan_create(&lp.o, s->attn, d, T, d, wo, 1, d, d, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, 0);
+        if (rc != SFS_OK) return rc;
+        const void *gu[2] = {m->w_gate[l], m->w_up[l]};
+        rc = gemm_plan_create(&lp.gate_up, s->h, d, T, d, gu, 2, ff, d, GEMM_SWIGLU, s->hid, ff, 0, 1.0f, nullptr, 0, 0, 0);
+        if (rc != SFS_OK) return rc;
+        const void *wd[1] = {m->w_down[l]};
+        rc = gemm_plan_create(&lp.down, s->hid, ff, T, ff, wd, 1, d, ff, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, 0);
+        if (rc != SFS_OK) return rc;
+    }
+    rc = attn_plan_create(&s->attn_plan, s->qk, 2 * d, s->vt, T, s->attn, d, B, S, c.n_heads, c.head_dim);
+    if (rc != SFS_OK) return rc;
+    const void *lm[1] = {m->lm_head};
+    rc = gemm_plan_create(&s->lm_plan, s->hfin, d, T, d, lm, 1, c.vocab, d, GEMM_STORE, s->logits, c.vocab, 0, c.logit_scale,
+                          nullptr, 0, 0, 0);
+    if (rc != SFS_OK) return rc;
+    s->plan_B = B; s->plan_S = S;
+    return SFS_OK;
+}
+
+// the transformer body: tokens -> residual stream x [T, d]
+static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t S, const int32_t *d_active, cudaStream_t st)
+{
+    const sfs_model *m = s->model;
+    const sfs_config &c = m->cfg;
+    const int T = B * S, d = c.d_model;
+    int32_t *err = device_status_word();
+    SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
+    int32_t rc;
+    if ((rc = launch_embed(d_tokens, m->tok_emb, s->x, T, d, c.vocab, st)) != SFS_OK) return rc;
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerPlans &lp = s->layer_plans[l];
+        if ((rc = launch_rmsnorm(s->x, m->attn_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st)) != SFS_OK) return rc;
+        if ((rc = gemm_launch(lp.qkv, nullptr, d_active, err, st)) != SFS_OK) return rc;
+        if ((rc = launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, st)) != SFS_OK) return rc;
+        if ((rc = attn_launch(s->attn_plan, d_active, err, st)) != SFS_OK) return rc;
+        if ((rc = gemm_launch(lp.o, nullptr, d_active, err, st)) != SFS_OK) return rc;
+        if ((rc = launch_rmsnorm(s->x, m->mlp_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st)) != SFS_OK) return rc;
+        if ((rc = gemm_launch(lp.gate_up, nullptr, d_active, err, st)) != SFS_OK) return rc;
+        if ((rc = gemm_launch(lp.down, nullptr, d_active, err, st)) != SFS_OK) return rc;
+    }
+    return SFS_OK;
+}
+
+__global__ void generate_init_kernel(const int32_t *prompt, int32_t *tokens, uint8_t *mask, int32_t *rows, int32_t *ctrl,
+                                     int32_t *host_active, unsigned long long *pos_sq, int B, int P, int L, int mask_id)
+{
+    const int S = P + L;
+    const long long n = (long long)B * S;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const int b = (int)(i / S), pos = (int)(i % S);
+        tokens[i] = pos < P ? prompt[(long long)b * P + pos] : mask_id;
+        mask[i] = pos < P ? 0 : 1;
+        pos_sq[i] = 0;
+        if (pos >= P) rows[(long long)b * L + (pos - P)] = (int)i;         // first step: every response row, sequence-major
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctrl[0] = B * L; ctrl[1] = 0; ctrl[2] = (L > 0) ? B : 0;
+        *host_active = (L > 0) ? B : 0;
+    }
+}
+
+__global__ void mirror_active_kernel(const int32_t *ctrl_active, int32_t *host_active) { *host_active = *ctrl_active; }
+
 }  // namespace sfs
 
 using namespace sfs;
@@ -64,6 +170,152 @@ const char *sfs_status_string(int32_t s)
         case SFS_ERR_MISSING_ROW: return "row statistics missing for a needed position";
         default: return "unknown status";
     }
+}
+
+int32_t sfs_check_device_status(void *stream)
+{
+    int32_t *err = device_status_word();
+    SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
+    SFS_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    int32_t h = 0;
+    SFS_CUDA(cudaMemcpy(&h, err, 4, cudaMemcpyDeviceToHost));
+    if (h != 0) {
+        cudaMemset(err, 0, 4);
+        set_error("a kernel reported device status %d (%s)", h, sfs_status_string(h));
+    }
+    return h;
+}
+
+// ---- model ----------------------------------------------------------------------------------------------
+int32_t sfs_model_create(const sfs_config *cfg, const sfs_weights *w, sfs_model **out)
+{
+    SFS_REQUIRE(cfg && w && out, SFS_ERR_INVALID_ARG, "model_create: NULL argument");
+    SFS_REQUIRE(cfg->n_layers >= 1 && cfg->d_model >= 8 && cfg->n_heads >= 1 && cfg->d_ff >= 8 && cfg->vocab >= 8,
+                SFS_ERR_INVALID_ARG, "model_create: sizes must be positive");
+    SFS_REQUIRE(cfg->head_dim == 64 || cfg->head_dim == 128, SFS_ERR_UNSUPPORTED, "head_dim %d (64 or 128 supported)", cfg->head_dim);
+    SFS_REQUIRE(cfg->n_heads * cfg->head_dim == cfg->d_model, SFS_ERR_INVALID_ARG, "n_heads * head_dim != d_model");
+    SFS_REQUIRE((cfg->d_model % 128) == 0, SFS_ERR_UNSUPPORTED, "d_model %d must be a multiple of 128", cfg->d_model);
+    SFS_REQUIRE((cfg->d_ff % 8) == 0 && (cfg->vocab % 8) == 0, SFS_ERR_UNSUPPORTED, "d_ff and vocab must be multiples of 8");
+    SFS_REQUIRE(cfg->vocab < (1 << 19), SFS_ERR_UNSUPPORTED, "vocab %d must be below 2^19", cfg->vocab);
+    SFS_REQUIRE(cfg->mask_id >= 0 && cfg->mask_id < cfg->vocab, SFS_ERR_INVALID_ARG, "mask_id outside the vocabulary");
+    SFS_REQUIRE(w->tok_emb && w->final_norm && w->lm_head && w->attn_norm && w->wq && w->wk && w->wv && w->wo &&
+                w->mlp_norm && w->w_gate && w->w_up && w->w_down, SFS_ERR_INVALID_ARG, "model_create: NULL weight table");
+    sfs_model *m = new (std::nothrow) sfs_model();
+    SFS_REQUIRE(m != nullptr, SFS_ERR_OOM, "host allocation failed");
+    m->cfg = *cfg;
+    m->tok_emb = w->tok_emb; m->final_norm = w->final_norm; m->lm_head = w->lm_head;
+    bool ok = aligned_to(w->tok_emb, 16) && aligned_to(w->final_norm, 16) && aligned_to(w->lm_head, 16);
+    for (int l = 0; l < cfg->n_layers; ++l) {
+        const void *ps[9] = {w->attn_norm[l], w->wq[l], w->wk[l], w->wv[l], w->wo[l], w->mlp_norm[l], w->w_gate[l], w->w_up[l], w->w_down[l]};
+        for (const void *p : ps) ok = ok && p != nullptr && aligned_to(p, 16);
+        m->attn_norm.push_back(ps[0]); m->wq.push_back(ps[1]); m->wk.push_back(ps[2]); m->wv.push_back(ps[3]);
+        m->wo.push_back(ps[4]); m->mlp_norm.push_back(ps[5]); m->w_gate.push_back(ps[6]); m->w_up.push_back(ps[7]);
+        m->w_down.push_back(ps[8]);
+    }
+    if (!ok) { delete m; set_error("model_create: every weight pointer must be non-NULL and 16-byte aligned"); return SFS_ERR_INVALID_ARG; }
+    *out = m;
+    return SFS_OK;
+}
+
+int32_t sfs_model_destroy(sfs_model *m)
+{
+    delete m;
+    return SFS_OK;
+}
+
+// ---- sessions -------------------------------------------------------------------------------------------
+int32_t sfs_session_destroy(sfs_session *s)
+{
+    if (!s) return SFS_OK;
+    cudaDeviceSynchronize();
+    for (void *p : s->owned) cudaFree(p);
+    if (s->host_active) cudaFreeHost(s->host_active);
+    delete s;
+    return SFS_OK;
+}
+
+int32_t sfs_select_session_create(int32_t vocab, int32_t max_batch, int32_t max_seq, sfs_session **out)
+{
+    SFS_REQUIRE(out != nullptr, SFS_ERR_INVALID_ARG, "out is NULL");
+    SFS_REQUIRE(vocab >= 1 && vocab < (1 << 19), SFS_ERR_INVALID_ARG, "vocab %d outside [1, 2^19)", vocab);
+    SFS_REQUIRE(max_batch >= 1 && max_seq >= 1 && max_seq < (1 << 17) && (long long)max_batch * max_seq < (1ll << 30),
+                SFS_ERR_INVALID_ARG, "max_batch %d / max_seq %d out of range", max_batch, max_seq);
+    sfs_session *s = new (std::nothrow) sfs_session();
+    SFS_REQUIRE(s != nullptr, SFS_ERR_OOM, "host allocation failed");
+    s->max_batch = max_batch; s->max_seq = max_seq; s->vocab = vocab;
+    int32_t rc = session_alloc_select(s);
+    if (rc != SFS_OK) { sfs_session_destroy(s); return rc; }
+    SFS_CUDA(cudaDeviceSynchronize());
+    *out = s;
+    return SFS_OK;
+}
+
+int32_t sfs_session_create(sfs_model *m, int32_t max_batch, int32_t max_seq, sfs_session **out)
+{
+    SFS_REQUIRE(m && out, SFS_ERR_INVALID_ARG, "session_create: NULL argument");
+    SFS_REQUIRE(max_batch >= 1 && max_seq >= 8 && max_seq < (1 << 17) && (long long)max_batch * max_seq < (1ll << 24),
+                SFS_ERR_INVALID_ARG, "max_batch %d / max_seq %d out of range", max_batch, max_seq);
+    sfs_session *s = new (std::nothrow) sfs_session();
+    SFS_REQUIRE(s != nullptr, SFS_ERR_OOM, "host allocation failed");
+    s->model = m; s->max_batch = max_batch; s->max_seq = max_seq; s->vocab = m->cfg.vocab;
+    const sfs_config &c = m->cfg;
+    const size_t T = (size_t)max_batch * max_seq, d = c.d_model;
+    int32_t rc = session_alloc_select(s);
+    auto fail = [&](int32_t code) { sfs_session_destroy(s); return code; };
+    if (rc != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->x, T * d, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->h, T * d, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->qk, T * 2 * d, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->vt, T * d, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->attn, T * d, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->hid, T * (size_t)c.d_ff, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->hfin, T * d, true)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->logits, T * (size_t)c.vocab, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->rope_table, (size_t)max_seq * (c.head_dim / 2), false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->tokens, T, true)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->mask, T, true)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->state, (size_t)max_batch, true)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->rows[0], T, true)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->rows[1], T, true)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->ctrl, 16, true)) != SFS_OK) return fail(rc);
+    if (cudaHostAlloc(reinterpret_cast<void **>(&s->host_active), 64, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer(reinterpret_cast<void **>(&s->host_active_dev), s->host_active, 0) != cudaSuccess) {
+        set_error("pinned host allocation failed");
+        return fail(SFS_ERR_OOM);
+    }
+    *s->host_active = 0;
+    if ((rc = launch_rope_table(s->rope_table, max_seq, c.head_dim, c.rope_theta, 0)) != SFS_OK) return fail(rc);
+    if (device_status_word() == nullptr) { set_error("cannot allocate the device status word"); return fail(SFS_ERR_OOM); }
+    if (cudaDeviceSynchronize() != cudaSuccess) { set_error("device synchronisation failed after session set-up"); return fail(SFS_ERR_CUDA); }
+    *out = s;
+    return SFS_OK;
+}
+
+// ---- single steps ---------------------------------------------------------------------------------------
+int32_t sfs_forward(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t S,
+                    const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
+                    void *d_logits, int32_t logits_dtype, void *stream)
+{
+    SFS_REQUIRE(s && s->model, SFS_ERR_INVALID_ARG, "forward: needs a session created from a model");
+    SFS_REQUIRE(d_tokens && d_logits, SFS_ERR_INVALID_ARG, "forward: NULL device pointer");
+    SFS_REQUIRE(B >= 1 && B <= s->max_batch && S >= 8 && S <= s->max_seq, SFS_ERR_INVALID_ARG,
+                "forward: B=%d S=%d outside the session's limits (%d, %d)", B, S, s->max_batch, s->max_seq);
+    SFS_REQUIRE(max_rows >= 1 && max_rows <= B * S, SFS_ERR_INVALID_ARG, "forward: max_rows %d outside [1, B*S]", max_rows);
+    SFS_REQUIRE(logits_dtype == SFS_LOGITS_BF16 || logits_dtype == SFS_LOGITS_F32, SFS_ERR_INVALID_ARG, "logits_dtype %d", logits_dtype);
+    SFS_REQUIRE(d_rows != nullptr || (max_rows == B * S && d_n_rows == nullptr), SFS_ERR_INVALID_ARG,
+                "forward: without a row list all B*S rows are produced");
+    cudaStream_t st = (cudaStream_t)stream;
+    const sfs_config &c = s->model->cfg;
+    int32_t rc = session_plan(s, B, S);
+    if (rc != SFS_OK) return rc;
+    if ((rc = run_body(s, d_tokens, B, S, nullptr, st)) != SFS_OK) return rc;
+    if ((rc = launch_rmsnorm(s->x, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st)) != SFS_OK) return rc;
+    GemmPlan lm;
+    const void *lmw[1] = {s->model->lm_head};
+    rc = gemm_plan_create(&lm, s->hfin, c.d_model, max_rows, c.d_model, lmw, 1, c.vocab, c.d_model, GEMM_STORE, d_logits, c.vocab,
+                          logits_dtype == SFS_LOGITS_F32 ? 1 : 0, c.logit_scale, nullptr, 0, 0, 0);
+    if (rc != SFS_OK) return rc;
+    return gemm_launch(lm, d_n_rows, nullptr, device_status_word(), st);
 }
 
 int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
@@ -121,65 +373,119 @@ int32_t sfs_select(sfs_session *s, const void *d_logits, int32_t logits_dtype, i
     return launch_select(a, st);
 }
 
-}  // extern "C"
-
-// ---- sessions -------------------------------------------------------------------------------------------
-namespace sfs {
-template <typename T>
-static int32_t dev_alloc(sfs_session *s, T **out, size_t count, bool zero)
+// ---- the whole loop -------------------------------------------------------------------------------------
+int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, int32_t P, int32_t gen_len,
+                           const sfs_params *params, void *stream)
 {
-    void *p = nullptr;
-    SFS_CUDA(cudaMalloc(&p, count * sizeof(T) > 0 ? count * sizeof(T) : 16));
-    s->owned.push_back(p);
-    if (zero) SFS_CUDA(cudaMemset(p, 0, count * sizeof(T)));
-    *out = reinterpret_cast<T *>(p);
+    SFS_REQUIRE(s && s->model, SFS_ERR_INVALID_ARG, "generate: needs a session created from a model");
+    SFS_REQUIRE(B >= 1 && B <= s->max_batch && P >= 0 && gen_len >= 1 && P + gen_len <= s->max_seq, SFS_ERR_INVALID_ARG,
+                "generate: B=%d P=%d gen_len=%d outside the session's limits (%d, %d)", B, P, gen_len, s->max_batch, s->max_seq);
+    SFS_REQUIRE(P == 0 || d_prompt != nullptr, SFS_ERR_INVALID_ARG, "generate: d_prompt is NULL");
+    int32_t rc = check_params(params);
+    if (rc != SFS_OK) return rc;
+    const int S = P + gen_len;
+    if ((rc = session_plan(s, B, S)) != SFS_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    generate_init_kernel<<<64, 256, 0, st>>>(d_prompt, s->tokens, s->mask, s->rows[0], s->ctrl, s->host_active_dev, s->pos_sq,
+                                             B, P, gen_len, s->model->cfg.mask_id);
+    SFS_LAUNCH_CHECK();
+    if ((rc = launch_state_init(s->state, B, gen_len, *params, nullptr, st)) != SFS_OK) return rc;
+    s->gen_B = B; s->gen_P = P; s->gen_L = gen_len; s->gen_cur = 0; s->gen_steps = 0;
+    s->gen_max_steps = params->max_steps > 0 ? params->max_steps : gen_len;
+    s->gen_params = *params;
+    s->generating = true;
+    *s->host_active = B;
     return SFS_OK;
 }
-}  // namespace sfs
 
-extern "C" {
-
-static int32_t session_alloc_select(sfs_session *s)
+int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, int32_t max_trace_steps,
+                           void *d_logits_dump, int32_t *d_rows_dump, int32_t *d_n_rows_dump, void *stream)
 {
-    const size_t n = (size_t)s->max_batch * s->max_seq;
+    SFS_REQUIRE(s && s->model && s->generating, SFS_ERR_INVALID_ARG, "generate_steps: call sfs_generate_begin first");
+    SFS_REQUIRE(n_steps >= 0, SFS_ERR_INVALID_ARG, "generate_steps: n_steps %d", n_steps);
+    SFS_REQUIRE(d_logits_dump == nullptr || n_steps == 1, SFS_ERR_INVALID_ARG, "generate_steps: a logits dump takes exactly one step");
+    cudaStream_t st = (cudaStream_t)stream;
+    const sfs_config &c = s->model->cfg;
+    const int B = s->gen_B, P = s->gen_P, L = s->gen_L, S = P + L;
+    int32_t *err = device_status_word();
     int32_t rc;
-    if ((rc = dev_alloc(s, &s->pos_sq, n, true)) != SFS_OK) return rc;
-    if ((rc = dev_alloc(s, &s->pos_arg, n, true)) != SFS_OK) return rc;
-    if ((rc = dev_alloc(s, &s->seq_rows, n, true)) != SFS_OK) return rc;
-    if ((rc = dev_alloc(s, &s->seq_row_count, (size_t)s->max_batch, true)) != SFS_OK) return rc;
-    if ((rc = dev_alloc(s, &s->ticket, 4, true)) != SFS_OK) return rc;
+    for (int i = 0; i < n_steps; ++i) {
+        if (s->gen_steps >= s->gen_max_steps) break;                 // every sequence is done by construction
+        const int cur = s->gen_cur, nxt = cur ^ 1;
+        const int32_t *d_active = s->ctrl + 2;
+        const int32_t *rows = s->rows[cur], *n_rows = s->ctrl + cur;
+        if ((rc = run_body(s, s->tokens, B, S, d_active, st)) != SFS_OK) return rc;
+        if ((rc = launch_rmsnorm(s->x, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st)) != SFS_OK) return rc;
+        GemmPlan lm = s->lm_plan;
+        lm.args.M = B * L;
+        if ((rc = gemm_launch(lm, n_rows, d_active, err, st)) != SFS_OK) return rc;
+        if (d_logits_dump) {
+            SFS_CUDA(cudaMemcpyAsync(d_logits_dump, s->logits, (size_t)B * L * c.vocab * 2, cudaMemcpyDeviceToDevice, st));
+            if (d_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_rows_dump, rows, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
+            if (d_n_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_n_rows_dump, n_rows, 4, cudaMemcpyDeviceToDevice, st));
+        }
+        if ((rc = launch_row_stats(s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, nullptr, nullptr, nullptr,
+                                   s->pos_sq, s->pos_arg, st)) != SFS_OK) return rc;
+        SelectArgs a{};
+        a.tokens = s->tokens; a.mask = s->mask; a.B = B; a.S = S; a.P = P; a.L = L;
+        a.state = s->state; a.params = s->gen_params;
+        a.pos_sq = s->pos_sq; a.pos_arg = s->pos_arg;
+        a.seq_rows = s->seq_rows; a.seq_row_count = s->seq_row_count;
+        a.next_rows = s->rows[nxt]; a.next_n_rows = s->ctrl + nxt; a.n_active = s->ctrl + 2;
+        a.ticket = s->ticket;
+        a.trace = (d_trace && s->gen_steps < max_trace_steps) ? d_trace + (size_t)s->gen_steps * B * SFS_TRACE_INTS : nullptr;
+        if ((rc = launch_select(a, st)) != SFS_OK) return rc;
+        mirror_active_kernel<<<1, 1, 0, st>>>(s->ctrl + 2, s->host_active_dev);
+        SFS_LAUNCH_CHECK();
+        s->gen_cur = nxt;
+        s->gen_steps++;
+    }
     return SFS_OK;
 }
 
-int32_t sfs_session_destroy(sfs_session *s)
+int32_t sfs_generate_end(sfs_session *s, int32_t *d_out_tokens, sfs_state *d_state_out, int32_t *n_active,
+                         int32_t *steps_enqueued, void *stream)
 {
-    if (!s) return SFS_OK;
-    cudaDeviceSynchronize();
-    for (void *p : s->owned) cudaFree(p);
-    delete s;
+    SFS_REQUIRE(s && s->model && s->generating, SFS_ERR_INVALID_ARG, "generate_end: call sfs_generate_begin first");
+    cudaStream_t st = (cudaStream_t)stream;
+    const int B = s->gen_B, S = s->gen_P + s->gen_L;
+    if (d_out_tokens) SFS_CUDA(cudaMemcpyAsync(d_out_tokens, s->tokens, (size_t)B * S * 4, cudaMemcpyDeviceToDevice, st));
+    if (d_state_out) SFS_CUDA(cudaMemcpyAsync(d_state_out, s->state, (size_t)B * sizeof(sfs_state), cudaMemcpyDeviceToDevice, st));
+    std::vector<sfs_state> hs((size_t)B);
+    SFS_CUDA(cudaMemcpyAsync(hs.data(), s->state, (size_t)B * sizeof(sfs_state), cudaMemcpyDeviceToHost, st));
+    int32_t dev = sfs_check_device_status(stream);                 // synchronises
+    if (steps_enqueued) *steps_enqueued = s->gen_steps;
+    int act = 0, bad = SFS_OK;
+    for (const sfs_state &h : hs) {
+        if (!h.done && h.status == SFS_OK) act++;
+        if (h.status != SFS_OK && bad == SFS_OK) bad = h.status;
+    }
+    if (n_active) *n_active = act;
+    if (dev != SFS_OK) return dev;
+    if (bad != SFS_OK) { set_error("a sequence stopped with device status %d (%s)", bad, sfs_status_string(bad)); return bad; }
     return SFS_OK;
 }
 
-int32_t sfs_select_session_create(int32_t vocab, int32_t max_batch, int32_t max_seq, sfs_session **out)
+int32_t sfs_generate(sfs_session *s, const int32_t *d_prompt, int32_t B, int32_t P, int32_t gen_len,
+                     const sfs_params *params, int32_t *d_out_tokens, sfs_state *d_state_out,
+                     int32_t *d_trace, int32_t max_trace_steps, void *stream)
 {
-    SFS_REQUIRE(out != nullptr, SFS_ERR_INVALID_ARG, "out is NULL");
-    SFS_REQUIRE(vocab >= 1 && vocab < (1 << 19), SFS_ERR_INVALID_ARG, "vocab %d outside [1, 2^19)", vocab);
-    SFS_REQUIRE(max_batch >= 1 && max_seq >= 1 && max_seq < (1 << 17) && (long long)max_batch * max_seq < (1ll << 30),
-                SFS_ERR_INVALID_ARG, "max_batch %d / max_seq %d out of range", max_batch, max_seq);
-    sfs_session *s = new (std::nothrow) sfs_session();
-    SFS_REQUIRE(s != nullptr, SFS_ERR_OOM, "host allocation failed");
-    s->max_batch = max_batch; s->max_seq = max_seq; s->vocab = vocab;
-    int32_t rc = session_alloc_select(s);
-    if (rc != SFS_OK) { sfs_session_destroy(s); return rc; }
-    SFS_CUDA(cudaDeviceSynchronize());
-    *out = s;
+    int32_t rc = sfs_generate_begin(s, d_prompt, B, P, gen_len, params, stream);
+    if (rc != SFS_OK) return rc;
+    // Steps are enqueued ahead of the device; the pinned mirror of the active-sequence count stops the
+    // enqueueing soon after the last sequence finishes, and kernels of surplus steps exit at once.
+    while (s->gen_steps < s->gen_max_steps) {
+        if (*reinterpret_cast<volatile int32_t *>(s->host_active) == 0) break;
+        if ((rc = sfs_generate_steps(s, 1, d_trace, max_trace_steps, nullptr, nullptr, nullptr, stream)) != SFS_OK) return rc;
+    }
+    int32_t act = 0;
+    rc = sfs_generate_end(s, d_out_tokens, d_state_out, &act, nullptr, stream);
+    if (rc != SFS_OK) return rc;
+    if (act != 0) { set_error("%d sequence(s) unfinished after %d steps", act, s->gen_steps); return SFS_ERR_STEP_LIMIT; }
     return SFS_OK;
 }
 
-}  // extern "C"
-
-extern "C" {
-
+// ---- building blocks ------------------------------------------------------------------------------------
 int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, void *d_C, int64_t ldc,
                    int32_t M, int32_t N, int32_t K, int32_t out_dtype, float scale, void *stream)
 {
@@ -192,21 +498,21 @@ int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, v
     const void *bs[1] = {d_B};
     int32_t rc = gemm_plan_create(&plan, d_A, lda, M, K, bs, 1, N, ldb, GEMM_STORE, d_C, ldc, out_dtype, scale, nullptr, 0, 0, 0);
     if (rc != SFS_OK) return rc;
-    return gemm_launch(plan, nullptr, err, (cudaStream_t)stream);
+    return gemm_launch(plan, nullptr, nullptr, err, (cudaStream_t)stream);
 }
 
-int32_t sfs_check_device_status(void *stream)
+int32_t sfs_attention(const void *d_qk, const void *d_vt, void *d_out, int32_t B, int32_t S,
+                      int32_t n_heads, int32_t head_dim, void *stream)
 {
+    SFS_REQUIRE(d_qk && d_vt && d_out, SFS_ERR_INVALID_ARG, "attention: NULL pointer");
+    SFS_REQUIRE(B >= 1 && S >= 8 && n_heads >= 1, SFS_ERR_INVALID_ARG, "attention: bad sizes");
     int32_t *err = device_status_word();
     SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
-    SFS_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
-    int32_t h = 0;
-    SFS_CUDA(cudaMemcpy(&h, err, 4, cudaMemcpyDeviceToHost));
-    if (h != 0) {
-        cudaMemset(err, 0, 4);
-        set_error("a kernel reported device status %d (%s)", h, sfs_status_string(h));
-    }
-    return h;
+    const int d = n_heads * head_dim;
+    AttnPlan plan;
+    int32_t rc = attn_plan_create(&plan, d_qk, 2 * d, d_vt, (int64_t)B * S, d_out, d, B, S, n_heads, head_dim);
+    if (rc != SFS_OK) return rc;
+    return attn_launch(plan, nullptr, err, (cudaStream_t)stream);
 }
 
 }  // extern "C"

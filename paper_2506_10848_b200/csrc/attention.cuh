@@ -1,0 +1,31 @@
+// Internal interface of the tcgen05 attention kernel.
+#pragma once
+#include "sfs_common.cuh"
+#include <cuda.h>
+#include <string.h>
+#include <math.h>
+
+namespace sfs {
+
+struct AttnArgs {
+    int B, S, n_heads, d_model;
+    float scale_log2;                  // log2(e) / sqrt(head_dim)
+    __nv_bfloat16 *out; long long ld_out;
+    int32_t *err;
+    const int32_t *d_active;           // optional: the kernel does nothing when *d_active == 0
+};
+
+struct AttnPlan {
+    CUtensorMap tmQK, tmVt;
+    AttnArgs args;
+    int head_dim;
+};
+
+// qkv: [B*S, >= 2*d] bf16 rows (q at columns [0, d), k at [d, 2d), RoPE applied), ld_qkv elements between rows;
+// vt:  [d, B*S] bf16 (V transposed: feature-major), ld_vt elements between feature rows;
+// out: [B*S, d] bf16.
+int32_t attn_plan_create(AttnPlan *p, const void *qkv, int64_t ld_qkv, const void *vt, int64_t ld_vt,
+                         void *out, int64_t ld_out, int32_t B, int32_t S, int32_t n_heads, int32_t head_dim);
+int32_t attn_launch(const AttnPlan &p, const int32_t *d_active, int32_t *err, cudaStream_t stream);
+
+}  // namespace sfs

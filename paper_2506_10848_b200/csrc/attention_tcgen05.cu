@@ -1,0 +1,280 @@
+// Bidirectional (unmasked) multi-head attention of the mask predictor: out = softmax(q k^T / sqrt(dh)) v
+// over all S positions of the same sequence.
+//
+// One CTA owns 128 query rows of one (sequence, head).  Warp 0 streams K tiles [128 keys x dh] and V^T
+// tiles [dh x 128 keys] through a two-stage TMA ring, warp 1 issues tcgen05.mma for S = Q K^T (accumulator
+// in tensor memory) and for O_j = P V_j, warps 2-5 (one thread per query row) run the online softmax in fp32
+// on S read back with tcgen05.ld, write P as bf16 into shared memory in the 128-byte-swizzled K-major
+// layout the next MMA consumes, and fold each O_j into a register accumulator with the running rescale.
+// V is consumed transposed (features x tokens); the QKV projection's epilogue writes it that way.
+#include "sfs_common.cuh"
+#include "tc05.cuh"
+#include "attention.cuh"
+
+namespace sfs {
+namespace {
+
+constexpr int kAttnThreads = 192;
+constexpr int QT = 128;                 // query rows per CTA
+constexpr int KT = 128;                 // keys per tile
+constexpr int KV_STAGES = 2;
+
+template <int DH>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant__ CUtensorMap tmVt, AttnArgs a)
+{
+    constexpr int KB = DH / 64;                          // 64-element K-blocks along the head dimension
+    constexpr int Q_BYTES = QT * DH * 2;
+    constexpr int K_BYTES = KT * DH * 2;
+    constexpr int V_BYTES = DH * KT * 2;
+    constexpr int P_BYTES = QT * KT * 2;
+    constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
+    constexpr uint32_t TMEM_COLS = (KT + DH) <= 256 ? 256 : 512;
+
+    if (a.d_active && *a.d_active == 0) return;          // nothing left to decode: uniform early exit
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = smem, *sKV = smem + Q_BYTES, *sP = sKV + KV_STAGES * STAGE_BYTES;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sP + P_BYTES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * KV_STAGES + 4);
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q0 = blockIdx.x * QT, h = blockIdx.y, b = blockIdx.z;
+    const int S = a.S, d = a.d_model;
+    const int tok0 = b * S;                                // first token of this sequence
+    const int nkv = (S + KT - 1) / KT;
+
+    const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * KV_STAGES;
+    const uint32_t bar_q = bar_empty + 8 * KV_STAGES, bar_s = bar_q + 8, bar_p = bar_q + 16, bar_o = bar_q + 24;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < KV_STAGES; ++s) { tc::mbar_init(bar_full + 8 * s, 1); tc::mbar_init(bar_empty + 8 * s, 1); }
+        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_s, 1); tc::mbar_init(bar_p, 128); tc::mbar_init(bar_o, 1);
+        s_abort = 0;
+        tc::mbar_init_fence();
+    }
+    if (warp == 1) { tc::tmem_alloc(tc::smem_u32(tmem_slot), TMEM_COLS); tc::tmem_relinquish(); }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
+    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + KT;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- TMA producer: Q once, then K / V^T tiles
+            tc::mbar_expect_tx(bar_q, Q_BYTES);
+#pragma unroll
+            for (int kb = 0; kb < KB; ++kb)
+                tc::tma_load_2d(tc::smem_u32(sQ) + kb * (QT * 128), &tmQK, h * DH + kb * 64, tok0 + q0, bar_q);
+            int issued = 0;
+            for (int j = 0; j < nkv; ++j) {
+                const int s = j % KV_STAGES;
+                const uint32_t ph = (uint32_t)(j / KV_STAGES) & 1u;
+                if (!tc::mbar_wait(bar_empty + 8 * s, ph ^ 1u, &s_abort)) break;
+                const uint32_t sk = tc::smem_u32(sKV) + s * STAGE_BYTES, sv = sk + K_BYTES;
+                tc::mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb)
+                    tc::tma_load_2d(sk + kb * (KT * 128), &tmQK, d + h * DH + kb * 64, tok0 + j * KT, bar_full + 8 * s);
+#pragma unroll
+                for (int kb = 0; kb < KT / 64; ++kb)
+                    tc::tma_load_2d(sv + kb * (DH * 128), &tmVt, tok0 + j * KT + kb * 64, h * DH, bar_full + 8 * s);
+                issued = j + 1;
+            }
+            if (s_abort) {
+                for (int j = max(0, issued - KV_STAGES); j < issued; ++j) {
+                    const uint32_t bar = bar_full + 8 * (j % KV_STAGES), ph = (uint32_t)(j / KV_STAGES) & 1u;
+                    for (int i = 0; i < (1 << 16) && !tc::mbar_try(bar, ph); ++i) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer
+            constexpr uint32_t idesc_s = tc::idesc_bf16_f32(QT, KT);
+            constexpr uint32_t idesc_o = tc::idesc_bf16_f32(QT, DH);
+            auto issue_S = [&](int s) {
+                const uint32_t sk = tc::smem_u32(sKV) + s * STAGE_BYTES;
+#pragma unroll
+                for (int kb = 0; kb < KB; ++kb) {
+                    const uint64_t dq = tc::smem_desc_sw128(tc::smem_u32(sQ) + kb * (QT * 128));
+                    const uint64_t dk = tc::smem_desc_sw128(sk + kb * (KT * 128));
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc::mma_bf16(tmem_S, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, (kb | kk) != 0 ? 1u : 0u);
+                }
+                tc::mma_commit(bar_s);
+            };
+            bool ok = tc::mbar_wait(bar_q, 0, &s_abort);
+            for (int j = 0; j < nkv && ok; ++j) {
+                const int s = j % KV_STAGES;
+                if (j == 0) {
+                    ok = tc::mbar_wait(bar_full + 8 * s, 0, &s_abort);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    issue_S(s);
+                }
+                ok = tc::mbar_wait(bar_p, (uint32_t)j & 1u, &s_abort);       // P_j is in shared memory, S_j has been read
+                if (!ok) break;
+                tc::tc_fence_after();
+                const uint32_t sv = tc::smem_u32(sKV) + s * STAGE_BYTES + K_BYTES;
+#pragma unroll
+                for (int kb = 0; kb < KT / 64; ++kb) {
+                    const uint64_t dp = tc::smem_desc_sw128(tc::smem_u32(sP) + kb * (QT * 128));
+                    const uint64_t dv = tc::smem_desc_sw128(sv + kb * (DH * 128));
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc::mma_bf16(tmem_O, dp + (uint64_t)(kk * 2), dv + (uint64_t)(kk * 2), idesc_o, (kb | kk) != 0 ? 1u : 0u);
+                }
+                tc::mma_commit(bar_o);
+                tc::mma_commit(bar_empty + 8 * s);
+                if (j + 1 < nkv) {
+                    const int s1 = (j + 1) % KV_STAGES;
+                    ok = tc::mbar_wait(bar_full + 8 * s1, (uint32_t)((j + 1) / KV_STAGES) & 1u, &s_abort);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    issue_S(s1);
+                }
+            }
+        }
+    } else {
+        // ---------------- online softmax + output accumulation: thread = query row
+        const int qd = warp & 3;
+        const int row = qd * 32 + lane;
+        const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
+        const float c = a.scale_log2;                      // log2(e) / sqrt(dh)
+        float m = -INFINITY, l = 0.f;
+        float acc[DH];
+#pragma unroll
+        for (int i = 0; i < DH; ++i) acc[i] = 0.f;
+        bool ok = true;
+        for (int j = 0; j < nkv && ok; ++j) {
+            ok = tc::mbar_wait(bar_s, (uint32_t)j & 1u, &s_abort);
+            if (!ok) break;
+            tc::tc_fence_after();
+            const int valid = min(KT, S - j * KT);         // keys of this tile that belong to the sequence
+            float mx = -INFINITY;
+#pragma unroll
+            for (int cc = 0; cc < KT / 32; ++cc) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_S + lane_off + cc * 32, v);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (cc * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+            }
+            const float m_new = fmaxf(m, mx);
+            const float alpha = exp2f((m - m_new) * c);
+            const float mc = m_new * c;
+            float lsum = 0.f;
+#pragma unroll
+            for (int cc = 0; cc < KT / 32; ++cc) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_S + lane_off + cc * 32, v);
+                tc::tmem_ld_wait();
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float p0 = (cc * 32 + 2 * i < valid) ? exp2f(fmaf(__uint_as_float(v[2 * i]), c, -mc)) : 0.f;
+                    const float p1 = (cc * 32 + 2 * i + 1 < valid) ? exp2f(fmaf(__uint_as_float(v[2 * i + 1]), c, -mc)) : 0.f;
+                    lsum += p0 + p1;
+                    __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
+                    pk[i] = *reinterpret_cast<uint32_t *>(&hh);
+                }
+                // keys cc*32 .. cc*32+31 of this row: K-block cc/2, 16-byte chunks (cc%2)*4 .. +3, swizzled by row
+                uint8_t *prow = sP + (cc >> 1) * (QT * 128) + row * 128;
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    const int chunk = ((cc & 1) * 4 + q4) ^ (row & 7);
+                    *reinterpret_cast<uint4 *>(prow + chunk * 16) = make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
+                }
+            }
+            l = l * alpha + lsum;
+            m = m_new;
+            tc::fence_proxy_async_smem();                  // P visible to the tensor core's shared-memory reads
+            tc::tc_fence_before();
+            tc::mbar_arrive(bar_p);
+            ok = tc::mbar_wait(bar_o, (uint32_t)j & 1u, &s_abort);
+            if (!ok) break;
+            tc::tc_fence_after();
+#pragma unroll
+            for (int cc = 0; cc < DH / 32; ++cc) {
+                uint32_t v[32];
+                tc::tmem_ld32(tmem_O + lane_off + cc * 32, v);
+                tc::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) acc[cc * 32 + i] = fmaf(acc[cc * 32 + i], alpha, __uint_as_float(v[i]));
+            }
+            tc::tc_fence_before();
+        }
+        if (ok && !s_abort && q0 + row < S) {
+            const float inv = 1.0f / l;
+            __nv_bfloat16 *dst = a.out + (long long)(tok0 + q0 + row) * a.ld_out + h * DH;
+#pragma unroll
+            for (int i = 0; i < DH / 8; ++i) {
+                uint32_t o[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    __nv_bfloat162 hh = __floats2bfloat162_rn(acc[8 * i + 2 * t] * inv, acc[8 * i + 2 * t + 1] * inv);
+                    o[t] = *reinterpret_cast<uint32_t *>(&hh);
+                }
+                reinterpret_cast<uint4 *>(dst)[i] = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+        }
+    }
+
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, TMEM_COLS); }
+    if (threadIdx.x == 0 && s_abort && a.err) atomicExch(a.err, SFS_ERR_TIMEOUT);
+}
+
+template <int DH>
+int32_t launch_dh(const AttnPlan &p, const int32_t *d_active, int32_t *err, cudaStream_t stream)
+{
+    constexpr size_t smem = (size_t)QT * DH * 2 + KV_STAGES * (size_t)(KT * DH * 2 + DH * KT * 2) + QT * KT * 2
+                          + (2 * KV_STAGES + 4) * 8 + 16 + 1024;
+    static bool configured = false;
+    if (!configured) {
+        SFS_CUDA(cudaFuncSetAttribute(attention_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured = true;
+    }
+    AttnArgs a = p.args;
+    a.err = err; a.d_active = d_active;
+    dim3 grid((unsigned)((a.S + QT - 1) / QT), (unsigned)a.n_heads, (unsigned)a.B);
+    attention_kernel<DH><<<grid, kAttnThreads, smem, stream>>>(p.tmQK, p.tmVt, a);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+}  // namespace
+
+int32_t attn_plan_create(AttnPlan *p, const void *qkv, int64_t ld_qkv, const void *vt, int64_t ld_vt,
+                         void *out, int64_t ld_out, int32_t B, int32_t S, int32_t n_heads, int32_t head_dim)
+{
+    SFS_REQUIRE(head_dim == 64 || head_dim == 128, SFS_ERR_UNSUPPORTED, "attention: head_dim %d (64 or 128 supported)", head_dim);
+    SFS_REQUIRE((S % 8) == 0, SFS_ERR_UNSUPPORTED, "attention: sequence length %d must be a multiple of 8", S);
+    SFS_REQUIRE(aligned_to(out, 16) && (ld_out % 8) == 0, SFS_ERR_INVALID_ARG, "attention: output must be 16-byte aligned");
+    memset(p, 0, sizeof(*p));
+    const int d = n_heads * head_dim;
+    int32_t rc = make_tmap_bf16(&p->tmQK, qkv, (uint64_t)B * S, (uint64_t)2 * d, (uint64_t)ld_qkv, 128);
+    if (rc != SFS_OK) return rc;
+    rc = make_tmap_bf16(&p->tmVt, vt, (uint64_t)d, (uint64_t)B * S, (uint64_t)ld_vt, (uint32_t)head_dim);
+    if (rc != SFS_OK) return rc;
+    AttnArgs &a = p->args;
+    a.B = B; a.S = S; a.n_heads = n_heads; a.d_model = d;
+    a.scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
+    a.out = reinterpret_cast<__nv_bfloat16 *>(out); a.ld_out = ld_out;
+    p->head_dim = head_dim;
+    return SFS_OK;
+}
+
+int32_t attn_launch(const AttnPlan &p, const int32_t *d_active, int32_t *err, cudaStream_t stream)
+{
+    if (p.head_dim == 128) return launch_dh<128>(p, d_active, err, stream);
+    return launch_dh<64>(p, d_active, err, stream);
+}
+
+}  // namespace sfs

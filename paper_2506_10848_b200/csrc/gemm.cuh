@@ -21,6 +21,7 @@ struct GemmArgs {
     __nv_bfloat16 *vt; long long ldvt; int vt_col0;
     int tiles_per_map;
     int32_t *err;            // device status word, set to SFS_ERR_TIMEOUT if a bounded wait gives up
+    const int32_t *d_active; // optional: the kernel does nothing when *d_active == 0
 };
 
 struct GemmPlan {
@@ -35,6 +36,6 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
                          const void *const *Bs, int32_t n_maps, int32_t n_per_map, int64_t ldb,
                          int32_t mode, void *C, int64_t ldc, int32_t out_f32, float scale,
                          __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, int32_t force_bn);
-int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, int32_t *err, cudaStream_t stream);
+int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream);
 
 }  // namespace sfs

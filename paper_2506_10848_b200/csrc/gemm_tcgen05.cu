@@ -70,6 +70,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     constexpr int HALF = BN / 2;
 
+    if (g.d_active && *g.d_active == 0) return;             // nothing left to decode: uniform early exit
     const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
     const int m_tile = blockIdx.x, n_tile = blockIdx.y;
     const int m0 = m_tile * BM;
@@ -256,7 +257,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 }
 
 template <int BN, int STAGES>
-int32_t launch_cfg(const GemmPlan &p, const int32_t *d_m, int32_t *err, cudaStream_t stream)
+int32_t launch_cfg(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
     constexpr size_t smem = (size_t)STAGES * (A_BYTES + BN * BK * 2) + (2 * STAGES + 1) * 8 + 16 + 1024;
     static bool configured = false;
@@ -265,7 +266,7 @@ int32_t launch_cfg(const GemmPlan &p, const int32_t *d_m, int32_t *err, cudaStre
         configured = true;
     }
     GemmArgs g = p.args;
-    g.d_m = d_m; g.err = err;
+    g.d_m = d_m; g.err = err; g.d_active = d_active;
     const int cols_per_tile = (g.mode == GEMM_SWIGLU) ? BN / 2 : BN;
     int n_tiles;
     if (g.mode == GEMM_SWIGLU || p.n_maps == 1) { n_tiles = (g.N + cols_per_tile - 1) / cols_per_tile; g.tiles_per_map = 0x3FFFFFFF; }
@@ -311,10 +312,10 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     return SFS_OK;
 }
 
-int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, int32_t *err, cudaStream_t stream)
+int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
-    if (p.bn == 256) return launch_cfg<256, 4>(p, d_m, err, stream);
-    return launch_cfg<128, 6>(p, d_m, err, stream);
+    if (p.bn == 256) return launch_cfg<256, 4>(p, d_m, d_active, err, stream);
+    return launch_cfg<128, 6>(p, d_m, d_active, err, stream);
 }
 
 }  // namespace sfs

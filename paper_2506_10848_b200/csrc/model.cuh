@@ -1,6 +1,8 @@
 // Model and session objects behind the opaque handles of the C ABI.
 #pragma once
 #include "sfs_common.cuh"
+#include "gemm.cuh"
+#include "attention.cuh"
 #include <vector>
 
 struct sfs_model {
@@ -8,12 +10,12 @@ struct sfs_model {
     // borrowed device pointers (copied pointer tables)
     const void *tok_emb, *final_norm, *lm_head;
     std::vector<const void *> attn_norm, wq, wk, wv, wo, mlp_norm, w_gate, w_up, w_down;
-    float2 *rope_table = nullptr;        // [max positions, head_dim/2] (cos, sin), owned
-    int32_t rope_positions = 0;
 };
 
+struct LayerPlans { sfs::GemmPlan qkv, o, gate_up, down; };
+
 struct sfs_session {
-    sfs_model *model = nullptr;          // may be NULL: a selection-only session
+    sfs_model *model = nullptr;          // NULL: a selection-only session
     int32_t max_batch = 0, max_seq = 0, vocab = 0;
     // selection scratch
     unsigned long long *pos_sq = nullptr;    // [max_batch*max_seq]
@@ -21,5 +23,32 @@ struct sfs_session {
     int32_t *seq_rows = nullptr;             // [max_batch*max_seq]
     int32_t *seq_row_count = nullptr;        // [max_batch]
     int32_t *ticket = nullptr;               // [1]
-    std::vector<void *> owned;               // everything to cudaFree at destroy
+    // forward workspace (model sessions only); T = max_batch*max_seq
+    float *x = nullptr;                      // [T, d] fp32 residual stream
+    __nv_bfloat16 *h = nullptr;              // [T, d] normalised activations
+    __nv_bfloat16 *qk = nullptr;             // [T, 2d] q | k
+    __nv_bfloat16 *vt = nullptr;             // [d, T] V transposed
+    __nv_bfloat16 *attn = nullptr;           // [T, d]
+    __nv_bfloat16 *hid = nullptr;            // [T, d_ff]
+    __nv_bfloat16 *hfin = nullptr;           // [T, d] gathered + normalised rows for the LM head
+    __nv_bfloat16 *logits = nullptr;         // [T, vocab]
+    float2 *rope_table = nullptr;            // [max_seq, head_dim/2]
+    // generation state
+    int32_t *tokens = nullptr;               // [T]
+    uint8_t *mask = nullptr;                 // [T]
+    sfs_state *state = nullptr;              // [max_batch]
+    int32_t *rows[2] = {nullptr, nullptr};   // [T] row lists of the current / next step
+    int32_t *ctrl = nullptr;                 // [0..1] row counts (double buffer), [2] active sequences
+    int32_t *host_active = nullptr;          // pinned, device-mapped mirror of ctrl[2]
+    int32_t *host_active_dev = nullptr;      // its device address
+    // plans for the shapes of the current call
+    int32_t plan_B = 0, plan_S = 0;
+    std::vector<LayerPlans> layer_plans;
+    sfs::AttnPlan attn_plan;
+    sfs::GemmPlan lm_plan;
+    // generation bookkeeping (host)
+    int32_t gen_B = 0, gen_P = 0, gen_L = 0, gen_cur = 0, gen_steps = 0, gen_max_steps = 0;
+    sfs_params gen_params;
+    bool generating = false;
+    std::vector<void *> owned;               // device allocations to free at destroy
 };
