@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the SlowFast denoising hot path at the LLaDA-8B shape.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload 8b|tiny]
+
+One "step" is one denoising step of the whole hot path: forward over prompt + partially masked response,
+LM head for the masked rows in scope, row statistics, SlowFast selection.  The workload is the
+LLaDA-8B-shaped random-init model, batch 1, 256 prompt ids + 256 masked positions (synthetic, seeded).
+K steps are timed with CUDA events on the launching stream after W warm-up steps; when a generation
+finishes inside the region the next one starts at once.  Prints one JSON line.
+
+Under torchrun (N > 1) every rank runs an independent replica on its own GPU (the path has no exchange
+step); the value is the sum of the ranks' tokens over the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"], bf16_tflops_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def step_flops(shape, T, S, rows):
+    """Algorithmic FLOPs of one denoising step: projections, attention, LM head for `rows` rows."""
+    d, ff, V, nl = shape.d_model, shape.d_ff, shape.vocab, shape.n_layers
+    gemm = 2.0 * T * (4 * d * d + 3 * d * ff) * nl
+    attn = 4.0 * T * S * d * nl
+    head = 2.0 * rows * d * V
+    return gemm, attn, head
+
+
+def step_bytes(shape, T, rows):
+    d, ff, V, nl = shape.d_model, shape.d_ff, shape.vocab, shape.n_layers
+    weights = 2.0 * ((4 * d * d + 3 * d * ff) * nl + d * V)
+    act = T * nl * (2 * d * 4 * 2 + 2 * d + 2 * 2 * d + 2 * d + 2 * d + 2 * 2 * ff)      # residual r/w (fp32), h, q|k, vT, attn, hidden w+r
+    logits = 2.0 * rows * V * 2
+    return weights + act + logits
+
+
+def run_ours(args, rank, world):
+    import torch
+    from paper_2506_10848_b200 import binding as sfs
+    from paper_2506_10848_b200 import workloads as W
+
+    local = int(os.environ.get("LOCAL_RANK", rank))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if args.workload == "tiny":
+        shape, P, L, B, name = W.TINY, 32, 64, 1, "tiny 2-layer d=256 model, batch 1, prompt 32 + 64 masked"
+    else:
+        shape, P, L, B, name = W.LLADA_8B, 256, 256, 1, "LLaDA-8B-shaped random-init model, batch 1, prompt 256 + 256 masked, no cache"
+    S = P + L
+    weights = W.model_weights(shape, seed=2 + rank, device=dev)
+    model = sfs.Model(shape, weights)
+    session = sfs.sfs_session_create(model, B, S)
+    params = sfs.Params.default()
+    prompt = W.prompt_ids(B, P, shape.vocab - 2, seed=2 + rank).to(dev)
+    out = torch.zeros((B, S), dtype=torch.int32, device=dev)
+    K, Wm = args.steps, args.warmup
+    trace = torch.zeros((K + Wm + 8, B, sfs.TRACE_INTS), dtype=torch.int32, device=dev)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps -------------------------
+    class Runner:
+        def __init__(self):
+            self.left = 0                         # steps left in the current generation (N = L at most)
+            self.gen_base = 0                     # trace row of the current generation's first step
+            self.total = 0
+
+        def step(self, n):
+            done = 0
+            while done < n:
+                if self.left == 0:
+                    sfs.sfs_generate_begin(session, prompt, B, P, L, params)
+                    self.left, self.gen_base = L, self.total
+                take = min(n - done, self.left)
+                sfs.sfs_generate_steps(session, take, trace[self.gen_base:], K + Wm + 8 - self.gen_base)
+                self.left -= take
+                done += take
+                self.total += take
+
+    r = Runner()
+    r.step(Wm)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    launches0 = sfs.sfs_profile(session, False, read=False)[2]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    r.step(K)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    launches = sfs.sfs_profile(session, False, read=False)[2] - launches0
+    sfs.sfs_check_device_status()
+    tr = trace[Wm:Wm + K].cpu()
+    tokens = int(tr[:, :, 5].sum())               # n_sel of every timed step
+    productive = int((tr[:, :, 5].sum(dim=1) > 0).sum())   # steps that unmasked something (all of them, normally)
+
+    # ---- per-kernel breakdown: the same steps again with CUDA events around every launch --------------
+    prof_steps = min(K, 16)
+    sfs.sfs_generate_begin(session, prompt, B, P, L, params)
+    sfs.sfs_profile(session, True, read=False)
+    sfs.sfs_generate_steps(session, prof_steps, None, 0)
+    ms_cls, cnt_cls, _ = sfs.sfs_profile(session, False, read=True)
+    gemm_classes = ["gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head"]
+    gemm_ms = sum(ms_cls[c] for c in gemm_classes)
+    gemm_launches = sum(cnt_cls[c] for c in gemm_classes)
+    T = B * S
+    # the first prof_steps steps of a generation see B*L, B*L-1, ... masked rows (one token per step here)
+    head_rows = sum(max(B * L - i, 1) for i in range(prof_steps)) / prof_steps
+    g_fl, a_fl, h_fl = step_flops(shape, T, S, head_rows)
+    gemm_tflops = (g_fl + h_fl) * prof_steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else None
+
+    # ---- end to end through sfs_generate with host buffers --------------------------------------------
+    e2e = None
+    if args.e2e:
+        host_prompt = prompt.cpu().pin_memory()
+        host_out = torch.zeros((B, S), dtype=torch.int32).pin_memory()
+        d_prompt = torch.zeros_like(prompt)
+        barrier()
+        t0 = time.perf_counter()
+        d_prompt.copy_(host_prompt, non_blocking=True)
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=dev)
+        sfs.sfs_generate(session, d_prompt, B, P, L, params, out, state)
+        host_out.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        gsteps = int(state[:, sfs.STATE_FIELDS.index("steps_done")].max())
+        e2e = {"value": B * L / (t1 - t0), "unit": "tokens/s", "h2d_bytes_per_step": B * P * 4 / max(gsteps, 1),
+               "d2h_bytes_per_step": B * S * 4 / max(gsteps, 1), "steps": gsteps, "seconds": t1 - t0,
+               "note": "one sfs_generate call: pinned host prompt -> device, full SlowFast loop, tokens -> pinned host"}
+
+    res = dict(productive=productive, ms=ms, tokens=tokens, launches=launches, clocks=clocks, ms_cls=ms_cls, cnt_cls=cnt_cls, gemm_ms=gemm_ms,
+               gemm_launches=gemm_launches, gemm_tflops=gemm_tflops, prof_steps=prof_steps, e2e=e2e, name=name, shape=shape,
+               T=T, S=S, B=B, L=L, P=P, head_rows=head_rows)
+    sfs.sfs_session_destroy(session)
+    model.close()
+    return res
+
+
+def oracle_sample(shape, P, L, seed=2):
+    """One bounded sample of the oracle at the 8B shape: ONE transformer layer over the full sequence, the LM
+    head and row statistics for 16 rows, and one selection step; extrapolated to a whole step."""
+    import numpy as np
+    from oracle import forward as F
+    from oracle import rowstats as RS
+    from oracle.scheduler import SlowFastParams, SlowFastState, rows_needed, slowfast_step
+    from paper_2506_10848_b200 import workloads as W
+
+    one = W.with_layers(shape, 1)
+    w = W.weights_to_numpy(W.model_weights(one, seed=seed), np.float32)
+    cfg = F.ModelConfig(**one.asdict())
+    tok = np.concatenate([W.prompt_ids(1, P, shape.vocab - 2, seed=seed).numpy(),
+                          np.full((1, L), shape.mask_id, np.int32)], axis=1)
+    head_rows = 16
+    t0 = time.perf_counter()
+    logits = F.forward(cfg, w, tok, rows=[(0, P + i) for i in range(head_rows)], dtype=np.float32)
+    t1 = time.perf_counter()
+    # time the LM head + row statistics separately on the same rows to extrapolate to L rows
+    hf = np.random.default_rng(0).standard_normal((head_rows, shape.d_model)).astype(np.float32)
+    t2 = time.perf_counter()
+    lg = hf @ w["lm_head"].T
+    st = RS.row_stats(np.ascontiguousarray(lg, dtype=np.float32))
+    t3 = time.perf_counter()
+    stt = SlowFastState.fresh(L, SlowFastParams())
+    rows = rows_needed(stt)
+    a = {i: int(st["argmax"][i % head_rows]) for i in rows}
+    sq = {i: int(st["sq"][i % head_rows]) for i in rows}
+    slowfast_step(stt, a, sq, SlowFastParams())
+    t4 = time.perf_counter()
+    per_row = (t3 - t2) / head_rows
+    layer_s = (t1 - t0) - (t3 - t2)                      # forward minus its own head
+    step_s = shape.n_layers * max(layer_s, 1e-6) + per_row * (L / 2.0) + (t4 - t3)
+    return dict(step_seconds=step_s, layer_seconds=layer_s, head_row_seconds=per_row, sample_seconds=t4 - t0)
+
+
+def run_reference(args, rank, world):
+    from paper_2506_10848_b200 import workloads as W
+    shape, P, L = (W.TINY, 32, 64) if args.workload == "tiny" else (W.LLADA_8B, 256, 256)
+    for _ in range(max(args.warmup, 0) and 1):
+        oracle_sample(shape, P, L)
+    ts = []
+    for _ in range(max(1, min(args.steps, 3))):
+        ts.append(oracle_sample(shape, P, L))
+    step_s = sorted(t["step_seconds"] for t in ts)[len(ts) // 2]
+    cores = os.cpu_count()
+    value = 1.0 / step_s                                   # one token per step on random-init logits
+    line = {"impl": "reference", "metric": "generated tokens/s at the LLaDA-8B shape (SlowFast, no cache)", "value": value,
+            "unit": "tokens/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": step_s * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "LLaDA-8B-shaped random-init model, batch 1, prompt 256 + 256 masked, no cache"
+                       if args.workload != "tiny" else "tiny"},
+            "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                             "sample": "per step: one of the 32 layers over all 512 tokens + LM head and row statistics for 16 rows "
+                                       "+ one selection step, in fp32 numpy; step time extrapolated as 32 x layer + L/2 rows x head"},
+            "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=128)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b", choices=["8b", "tiny"])
+    ap.add_argument("--no-e2e", dest="e2e", action="store_false")
+    ap.add_argument("--no-cpu-baseline", dest="cpu", action="store_false")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+
+    if args.impl == "reference":
+        if rank == 0:
+            run_reference(args, rank, world)
+        return
+
+    import torch
+    if world > 1:
+        torch.distributed.init_process_group("nccl")
+    import __graft_entry__ as entry
+    if rank == 0:
+        entry.build()
+    if world > 1:
+        torch.distributed.barrier()
+    res = run_ours(args, rank, world)
+
+    ms, tokens = res["ms"], res["tokens"]
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        k = torch.tensor([tokens, res["launches"]], dtype=torch.float64, device="cuda")
+        torch.distributed.all_reduce(k, op=torch.distributed.ReduceOp.SUM)
+        ms, tokens, launches = float(t[0]), int(k[0]), int(k[1])
+    else:
+        launches = res["launches"]
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    shape = res["shape"]
+    K = args.steps
+    ms_step = ms / K
+    g_fl, a_fl, h_fl = step_flops(shape, res["T"], res["S"], res["head_rows"])
+    step_roof_ms = max((g_fl + a_fl + h_fl) / (peaks["bf16_tflops"] * 1e12), step_bytes(shape, res["T"], res["head_rows"]) / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    roofline = {"bound": "tensor", "achieved": res["gemm_tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": (res["gemm_tflops"] / peaks["bf16_tflops_sustained"]) if res["gemm_tflops"] else None, "traffic": None,
+                "kernel": "gemm_kernel (tcgen05 projections: QKV, O, gate/up+SwiGLU, down, LM head)",
+                "peak_source": peaks["source"] + " (sustained cuBLAS bf16, kernel timed inside a long step)",
+                "launches_timed": res["gemm_launches"], "ms_timed": res["gemm_ms"], "steps_timed": res["prof_steps"]}
+    line = {"metric": "generated tokens/s at the LLaDA-8B shape (SlowFast, no cache)", "value": tokens / (ms * 1e-3),
+            "unit": "tokens/s", "n_gpus": world, "steps": K, "warmup": args.warmup, "ms_per_step": ms_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": res["name"], "l2": "inputs larger than L2 (16 GB of weights streamed every step)",
+                       "params": "tau_min 0.1, tau_high 0.85, K_max 8, W_hist 2, sigma2 1.0, k_slow = k_fast = 1, N = L"},
+            "tokens_unmasked": tokens, "productive_steps": res["productive"], "gpu_launches": launches, "clocks": res["clocks"],
+            "step_roofline_ms": step_roof_ms, "step_roofline_frac": step_roof_ms / ms_step,
+            "kernel_ms_per_step": {k: v / res["prof_steps"] for k, v in res["ms_cls"].items()},
+            "roofline": roofline, "e2e": res["e2e"]}
+    if args.cpu and world == 1:
+        from paper_2506_10848_b200 import workloads as W
+        P, L = (32, 64) if args.workload == "tiny" else (256, 256)
+        smp = oracle_sample(shape, P, L)
+        line["cpu_baseline"] = {"value": 1.0 / smp["step_seconds"], "unit": "tokens/s", "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"one of the {shape.n_layers} layers over all tokens + LM head and row statistics for 16 rows + one "
+                                          f"selection step (fp32 numpy, {smp['sample_seconds']:.1f} s); step time extrapolated as "
+                                          f"{shape.n_layers} x layer + L/2 rows x head; one token per step"}
+    print(json.dumps(line))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

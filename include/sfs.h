@@ -188,6 +188,30 @@ int32_t sfs_generate_steps(sfs_session *session, int32_t n_steps, int32_t *d_tra
 int32_t sfs_generate_end(sfs_session *session, int32_t *d_out_tokens, sfs_state *d_state_out,
                          int32_t *n_active, int32_t *steps_enqueued, void *stream);
 
+/* ---- instrumentation ------------------------------------------------------------------------------------ */
+
+/* Kernel classes of one denoising step, in launch order. */
+#define SFS_K_EMBED        0
+#define SFS_K_RMSNORM      1
+#define SFS_K_GEMM_QKV     2
+#define SFS_K_ROPE         3
+#define SFS_K_ATTENTION    4
+#define SFS_K_GEMM_O       5
+#define SFS_K_GEMM_GATE_UP 6
+#define SFS_K_GEMM_DOWN    7
+#define SFS_K_GEMM_LM_HEAD 8
+#define SFS_K_ROW_STATS    9
+#define SFS_K_SELECT       10
+#define SFS_K_CLASSES      11
+
+/* Per-kernel timing of a session's forward / generate launches.  First synchronises the device and, when the
+ * output pointers (HOST arrays of SFS_K_CLASSES entries) are not NULL, reports the milliseconds and launch
+ * counts gathered since the previous call, per kernel class; *total_launches (host, optional) receives the
+ * number of kernels the session has launched since it was created.  Then timing is switched on or off for the
+ * calls that follow: while on, every launch is bracketed by two CUDA events on its stream. */
+int32_t sfs_profile(sfs_session *session, int32_t enable, float *ms_per_class, int64_t *launches_per_class,
+                    int64_t *total_launches);
+
 /* ---- building blocks exposed for tests and measurements ------------------------------------------------- */
 
 /* C[M, N] = A[M, K] * B[N, K]^T, bf16 inputs, fp32 accumulation in tensor memory (tcgen05), output bf16

@@ -202,3 +202,17 @@ def sfs_generate_end(session, out_tokens=None, state_out=None, stream=None):
     na, ns = c_int32(0), c_int32(0)
     _check(lib().sfs_generate_end(session, _ptr(out_tokens), _ptr(state_out), byref(na), byref(ns), _stream(stream)))
     return na.value, ns.value
+
+
+K_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head",
+             "row_stats", "select"]
+
+
+def sfs_profile(session, enable, read=True):
+    """Returns (ms per class dict, launches per class dict, total launches) gathered since the previous call."""
+    n = len(K_CLASSES)
+    ms = (c_float * n)()
+    cnt = (c_int64 * n)()
+    tot = c_int64(0)
+    _check(lib().sfs_profile(session, c_int32(1 if enable else 0), ms if read else None, cnt if read else None, byref(tot)))
+    return dict(zip(K_CLASSES, list(ms))), dict(zip(K_CLASSES, list(cnt))), tot.value

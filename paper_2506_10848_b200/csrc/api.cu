@@ -104,6 +104,21 @@ static int32_t session_plan(sfs_session *s, int32_t B, int32_t S)
     return SFS_OK;
 }
 
+// Runs one launch; when profiling is on, brackets it with CUDA events tagged with the kernel class.
+template <typename F>
+static int32_t timed_launch(sfs_session *s, int cls, cudaStream_t st, F &&f)
+{
+    s->launches++;
+    if (!s->profile) return f();
+    sfs_session::Timed t; t.cls = cls;
+    SFS_CUDA(cudaEventCreate(&t.e0)); SFS_CUDA(cudaEventCreate(&t.e1));
+    SFS_CUDA(cudaEventRecord(t.e0, st));
+    int32_t rc = f();
+    SFS_CUDA(cudaEventRecord(t.e1, st));
+    s->timed.push_back(t);
+    return rc;
+}
+
 // the transformer body: tokens -> residual stream x [T, d]
 static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t S, const int32_t *d_active, cudaStream_t st)
 {
@@ -113,17 +128,17 @@ static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int3
     int32_t *err = device_status_word();
     SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
     int32_t rc;
-    if ((rc = launch_embed(d_tokens, m->tok_emb, s->x, T, d, c.vocab, st)) != SFS_OK) return rc;
+    if ((rc = timed_launch(s, SFS_K_EMBED, st, [&] { return launch_embed(d_tokens, m->tok_emb, s->x, T, d, c.vocab, st); })) != SFS_OK) return rc;
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerPlans &lp = s->layer_plans[l];
-        if ((rc = launch_rmsnorm(s->x, m->attn_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st)) != SFS_OK) return rc;
-        if ((rc = gemm_launch(lp.qkv, nullptr, d_active, err, st)) != SFS_OK) return rc;
-        if ((rc = launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, st)) != SFS_OK) return rc;
-        if ((rc = attn_launch(s->attn_plan, d_active, err, st)) != SFS_OK) return rc;
-        if ((rc = gemm_launch(lp.o, nullptr, d_active, err, st)) != SFS_OK) return rc;
-        if ((rc = launch_rmsnorm(s->x, m->mlp_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st)) != SFS_OK) return rc;
-        if ((rc = gemm_launch(lp.gate_up, nullptr, d_active, err, st)) != SFS_OK) return rc;
-        if ((rc = gemm_launch(lp.down, nullptr, d_active, err, st)) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, m->attn_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(lp.qkv, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch(s->attn_plan, d_active, err, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(lp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, m->mlp_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(lp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(lp.down, nullptr, d_active, err, st); })) != SFS_OK) return rc;
     }
     return SFS_OK;
 }
@@ -309,13 +324,13 @@ int32_t sfs_forward(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t 
     int32_t rc = session_plan(s, B, S);
     if (rc != SFS_OK) return rc;
     if ((rc = run_body(s, d_tokens, B, S, nullptr, st)) != SFS_OK) return rc;
-    if ((rc = launch_rmsnorm(s->x, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st)) != SFS_OK) return rc;
+    if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
     GemmPlan lm;
     const void *lmw[1] = {s->model->lm_head};
     rc = gemm_plan_create(&lm, s->hfin, c.d_model, max_rows, c.d_model, lmw, 1, c.vocab, c.d_model, GEMM_STORE, d_logits, c.vocab,
                           logits_dtype == SFS_LOGITS_F32 ? 1 : 0, c.logit_scale, nullptr, 0, 0, 0);
     if (rc != SFS_OK) return rc;
-    return gemm_launch(lm, d_n_rows, nullptr, device_status_word(), st);
+    return timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(lm, d_n_rows, nullptr, device_status_word(), st); });
 }
 
 int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
@@ -415,17 +430,18 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         const int32_t *d_active = s->ctrl + 2;
         const int32_t *rows = s->rows[cur], *n_rows = s->ctrl + cur;
         if ((rc = run_body(s, s->tokens, B, S, d_active, st)) != SFS_OK) return rc;
-        if ((rc = launch_rmsnorm(s->x, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st)) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
         GemmPlan lm = s->lm_plan;
         lm.args.M = B * L;
-        if ((rc = gemm_launch(lm, n_rows, d_active, err, st)) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(lm, n_rows, d_active, err, st); })) != SFS_OK) return rc;
         if (d_logits_dump) {
             SFS_CUDA(cudaMemcpyAsync(d_logits_dump, s->logits, (size_t)B * L * c.vocab * 2, cudaMemcpyDeviceToDevice, st));
             if (d_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_rows_dump, rows, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
             if (d_n_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_n_rows_dump, n_rows, 4, cudaMemcpyDeviceToDevice, st));
         }
-        if ((rc = launch_row_stats(s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, nullptr, nullptr, nullptr,
-                                   s->pos_sq, s->pos_arg, st)) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_ROW_STATS, st, [&] {
+                 return launch_row_stats(s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, nullptr, nullptr, nullptr,
+                                         s->pos_sq, s->pos_arg, st); })) != SFS_OK) return rc;
         SelectArgs a{};
         a.tokens = s->tokens; a.mask = s->mask; a.B = B; a.S = S; a.P = P; a.L = L;
         a.state = s->state; a.params = s->gen_params;
@@ -434,9 +450,10 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         a.next_rows = s->rows[nxt]; a.next_n_rows = s->ctrl + nxt; a.n_active = s->ctrl + 2;
         a.ticket = s->ticket;
         a.trace = (d_trace && s->gen_steps < max_trace_steps) ? d_trace + (size_t)s->gen_steps * B * SFS_TRACE_INTS : nullptr;
-        if ((rc = launch_select(a, st)) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_SELECT, st, [&] { return launch_select(a, st); })) != SFS_OK) return rc;
         mirror_active_kernel<<<1, 1, 0, st>>>(s->ctrl + 2, s->host_active_dev);
         SFS_LAUNCH_CHECK();
+        s->launches++;
         s->gen_cur = nxt;
         s->gen_steps++;
     }
@@ -482,6 +499,27 @@ int32_t sfs_generate(sfs_session *s, const int32_t *d_prompt, int32_t B, int32_t
     rc = sfs_generate_end(s, d_out_tokens, d_state_out, &act, nullptr, stream);
     if (rc != SFS_OK) return rc;
     if (act != 0) { set_error("%d sequence(s) unfinished after %d steps", act, s->gen_steps); return SFS_ERR_STEP_LIMIT; }
+    return SFS_OK;
+}
+
+// ---- instrumentation ------------------------------------------------------------------------------------
+int32_t sfs_profile(sfs_session *s, int32_t enable, float *ms_per_class, int64_t *launches_per_class, int64_t *total_launches)
+{
+    SFS_REQUIRE(s != nullptr, SFS_ERR_INVALID_ARG, "profile: session is NULL");
+    if (ms_per_class || launches_per_class) {
+        SFS_CUDA(cudaDeviceSynchronize());
+        for (int i = 0; i < SFS_K_CLASSES; ++i) { if (ms_per_class) ms_per_class[i] = 0.f; if (launches_per_class) launches_per_class[i] = 0; }
+        for (auto &t : s->timed) {
+            float ms = 0.f;
+            SFS_CUDA(cudaEventElapsedTime(&ms, t.e0, t.e1));
+            if (ms_per_class) ms_per_class[t.cls] += ms;
+            if (launches_per_class) launches_per_class[t.cls] += 1;
+        }
+    }
+    if (total_launches) *total_launches = s->launches;
+    for (auto &t : s->timed) { cudaEventDestroy(t.e0); cudaEventDestroy(t.e1); }
+    s->timed.clear();
+    s->profile = enable != 0;
     return SFS_OK;
 }
 

@@ -51,4 +51,9 @@ struct sfs_session {
     sfs_params gen_params;
     bool generating = false;
     std::vector<void *> owned;               // device allocations to free at destroy
+    // optional per-kernel-class timing (CUDA events around every launch) and launch counting
+    bool profile = false;
+    long long launches = 0;
+    struct Timed { int cls; cudaEvent_t e0, e1; };
+    std::vector<Timed> timed;
 };
