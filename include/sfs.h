@@ -165,6 +165,25 @@ int32_t sfs_select(sfs_session *session, const void *d_logits, int32_t logits_dt
                    int32_t *d_sel_count, int32_t *d_sel_pos, int32_t *d_sel_tok,
                    int32_t *d_next_rows, int32_t *d_next_n_rows, int32_t *d_trace, void *stream);
 
+/* The same step as sfs_select for callers that cannot allocate device memory (code running under a CUDA-graph
+ * capture or replay, serving loops that ban allocator calls, processes whose GPU memory belongs to another
+ * runtime's pool): no session is needed, because the scratch lives in a fixed array inside the library image.
+ * (The paper has no counterpart of this entry point; it exists for deployment only.)
+ *   Arguments as sfs_select, with `vocab` given explicitly.  Limits: B <= SFS_STATIC_MAX_BATCH sequences and
+ *   B*S <= SFS_STATIC_MAX_POSITIONS token positions, else SFS_ERR_UNSUPPORTED.  The array (about 260 KB) is held
+ *   by every GPU that loads the library until the process exits.  The call itself performs no cudaMalloc / cudaFree
+ *   and calls no allocating routine.  All calls share the array: it keeps the previous call's contents (the call
+ *   clears the parts that must start at zero), and calls whose kernels may overlap on the GPU race - run them one
+ *   after another.  The first call on each device looks up the array's address; make it before any stream capture. */
+#define SFS_STATIC_MAX_POSITIONS 16384
+#define SFS_STATIC_MAX_BATCH 64
+int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_t logits_dtype, int64_t ld,
+                          const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
+                          int32_t *d_tokens, uint8_t *d_mask, int32_t B, int32_t S, int32_t P,
+                          sfs_state *d_state, const sfs_params *params,
+                          int32_t *d_sel_count, int32_t *d_sel_pos, int32_t *d_sel_tok,
+                          int32_t *d_next_rows, int32_t *d_next_n_rows, int32_t *d_trace, void *stream);
+
 /* ---- the whole loop ------------------------------------------------------------------------------------ */
 
 /* Algorithm 1 for B independent sequences with a common prompt length P and response length gen_len:

@@ -216,3 +216,15 @@ def sfs_profile(session, enable, read=True):
     tot = c_int64(0)
     _check(lib().sfs_profile(session, c_int32(1 if enable else 0), ms if read else None, cnt if read else None, byref(tot)))
     return dict(zip(K_CLASSES, list(ms))), dict(zip(K_CLASSES, list(cnt))), tot.value
+
+
+STATIC_MAX_POSITIONS, STATIC_MAX_BATCH = 16384, 64
+
+
+def sfs_select_static(vocab, logits, logits_dtype, ld, rows, n_rows_dev, max_rows, tokens, mask, B, S, P, state, params,
+                      sel_count=None, sel_pos=None, sel_tok=None, next_rows=None, next_n_rows=None, trace=None, stream=None):
+    """sfs_select without a session: the scratch is a fixed array inside the library, so nothing is allocated."""
+    _check(lib().sfs_select_static(c_int32(vocab), _ptr(logits), c_int32(logits_dtype), c_int64(ld), _ptr(rows), _ptr(n_rows_dev),
+                                   c_int32(max_rows), _ptr(tokens), _ptr(mask), c_int32(B), c_int32(S), c_int32(P),
+                                   _ptr(state), byref(params), _ptr(sel_count), _ptr(sel_pos), _ptr(sel_tok),
+                                   _ptr(next_rows), _ptr(next_n_rows), _ptr(trace), _stream(stream)))
