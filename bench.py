@@ -107,6 +107,9 @@ def run_ours(args, rank, world):
         shape, P, L, B, name = W.TINY, 32, 64, 1, "tiny 2-layer d=256 model, batch 1, prompt 32 + 64 masked"
     else:
         shape, P, L, B, name = W.LLADA_8B, 256, 256, 1, "LLaDA-8B-shaped random-init model, batch 1, prompt 256 + 256 masked, no cache"
+    if args.layers:
+        shape = W.with_layers(shape, args.layers)
+        name += f" [reduced to {args.layers} layers: a profiling case, not a bench value]"
     S = P + L
     weights = W.model_weights(shape, seed=2 + rank, device=dev)
     model = sfs.Model(shape, weights)
@@ -268,6 +271,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=["8b", "tiny"])
+    ap.add_argument("--layers", type=int, default=0, help="keep only this many layers (small case for ncu captures)")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")
     ap.add_argument("--no-cpu-baseline", dest="cpu", action="store_false")
     args = ap.parse_args()
