@@ -82,23 +82,19 @@ static int32_t session_plan(sfs_session *s, int32_t B, int32_t S)
         LayerPlans &lp = s->layer_plans[l];
         const void *qkv[3] = {m->wq[l], m->wk[l], m->wv[l]};
         // q | k go row-major into qk [T, 2d]; the v columns (>= 2d) go transposed into vt [d, T]
-        rc = gemm_plan_create(&lp.qkv, s->h, d, T, d, qkv, 3, d, d, GEMM_STORE, s->qk, 2 * d, 0, 1.0f, s->vt, T, 2 * d, 0);
+        rc = gemm_plan_create(&lp.qkv, s->h, d, T, d, qkv, 3, d, d, GEMM_STORE, s->qk, 2 * d, 0, 1.0f, s->vt, T, 2 * d, nullptr);
         if (rc != SFS_OK) return rc;
         const void *wo[1] = {m->wo[l]};
-        rc = gemm_plan_create(&lp.o, s->attn, d, T, d, wo, 1, d, d, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, 0);
+        rc = gemm_plan_create(&lp.o, s->attn, d, T, d, wo, 1, d, d, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
         const void *gu[2] = {m->w_gate[l], m->w_up[l]};
-        rc = gemm_plan_create(&lp.gate_up, s->h, d, T, d, gu, 2, ff, d, GEMM_SWIGLU, s->hid, ff, 0, 1.0f, nullptr, 0, 0, 0);
+        rc = gemm_plan_create(&lp.gate_up, s->h, d, T, d, gu, 2, ff, d, GEMM_SWIGLU, s->hid, ff, 0, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
         const void *wd[1] = {m->w_down[l]};
-        rc = gemm_plan_create(&lp.down, s->hid, ff, T, ff, wd, 1, d, ff, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, 0);
+        rc = gemm_plan_create(&lp.down, s->hid, ff, T, ff, wd, 1, d, ff, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
     }
     rc = attn_plan_create(&s->attn_plan, s->qk, 2 * d, s->vt, T, s->attn, d, B, S, c.n_heads, c.head_dim);
-    if (rc != SFS_OK) return rc;
-    const void *lm[1] = {m->lm_head};
-    rc = gemm_plan_create(&s->lm_plan, s->hfin, d, T, d, lm, 1, c.vocab, d, GEMM_STORE, s->logits, c.vocab, 0, c.logit_scale,
-                          nullptr, 0, 0, 0);
     if (rc != SFS_OK) return rc;
     s->plan_B = B; s->plan_S = S;
     return SFS_OK;
@@ -328,7 +324,7 @@ int32_t sfs_forward(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t 
     GemmPlan lm;
     const void *lmw[1] = {s->model->lm_head};
     rc = gemm_plan_create(&lm, s->hfin, c.d_model, max_rows, c.d_model, lmw, 1, c.vocab, c.d_model, GEMM_STORE, d_logits, c.vocab,
-                          logits_dtype == SFS_LOGITS_F32 ? 1 : 0, c.logit_scale, nullptr, 0, 0, 0);
+                          logits_dtype == SFS_LOGITS_F32 ? 1 : 0, c.logit_scale, nullptr, 0, 0, nullptr);
     if (rc != SFS_OK) return rc;
     return timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(lm, d_n_rows, nullptr, device_status_word(), st); });
 }
@@ -401,6 +397,13 @@ int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, i
     const int S = P + gen_len;
     if ((rc = session_plan(s, B, S)) != SFS_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
+    {   // the LM head sees at most B * gen_len rows: plan it for that many, not for all B * S tokens
+        const sfs_config &c = s->model->cfg;
+        const void *lm[1] = {s->model->lm_head};
+        rc = gemm_plan_create(&s->lm_plan, s->hfin, c.d_model, B * gen_len, c.d_model, lm, 1, c.vocab, c.d_model, GEMM_STORE,
+                              s->logits, c.vocab, 0, c.logit_scale, nullptr, 0, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+    }
     generate_init_kernel<<<64, 256, 0, st>>>(d_prompt, s->tokens, s->mask, s->rows[0], s->ctrl, s->host_active_dev, s->pos_sq,
                                              B, P, gen_len, s->model->cfg.mask_id);
     SFS_LAUNCH_CHECK();
@@ -431,9 +434,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         const int32_t *rows = s->rows[cur], *n_rows = s->ctrl + cur;
         if ((rc = run_body(s, s->tokens, B, S, d_active, st)) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
-        GemmPlan lm = s->lm_plan;
-        lm.args.M = B * L;
-        if ((rc = timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(lm, n_rows, d_active, err, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(s->lm_plan, n_rows, d_active, err, st); })) != SFS_OK) return rc;
         if (d_logits_dump) {
             SFS_CUDA(cudaMemcpyAsync(d_logits_dump, s->logits, (size_t)B * L * c.vocab * 2, cudaMemcpyDeviceToDevice, st));
             if (d_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_rows_dump, rows, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
@@ -534,7 +535,7 @@ int32_t sfs_linear(const void *d_A, int64_t lda, const void *d_B, int64_t ldb, v
     SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
     GemmPlan plan;
     const void *bs[1] = {d_B};
-    int32_t rc = gemm_plan_create(&plan, d_A, lda, M, K, bs, 1, N, ldb, GEMM_STORE, d_C, ldc, out_dtype, scale, nullptr, 0, 0, 0);
+    int32_t rc = gemm_plan_create(&plan, d_A, lda, M, K, bs, 1, N, ldb, GEMM_STORE, d_C, ldc, out_dtype, scale, nullptr, 0, 0, nullptr);
     if (rc != SFS_OK) return rc;
     return gemm_launch(plan, nullptr, nullptr, err, (cudaStream_t)stream);
 }

@@ -19,7 +19,12 @@ struct GemmArgs {
     float scale;
     void *C; long long ldc;
     __nv_bfloat16 *vt; long long ldvt; int vt_col0;
-    int tiles_per_map;
+    int tiles_per_map;       // column tiles per B matrix (concatenated outputs)
+    int n_per_map;           // rows of each B matrix
+    int bn, stages;          // tile width (multiple of 16, <= 256) and depth of the shared-memory ring
+    int mb;                  // 256-row blocks per tile (1 or 2)
+    int n_col_tiles;         // column tiles over all B matrices
+    int acc_bufs;            // accumulator buffers in tensor memory (2 when they fit: epilogue overlaps the next tile)
     int32_t *err;            // device status word, set to SFS_ERR_TIMEOUT if a bounded wait gives up
     const int32_t *d_active; // optional: the kernel does nothing when *d_active == 0
 };
@@ -30,12 +35,15 @@ struct GemmPlan {
     int bn, n_maps, n_per_map;
 };
 
+// Optional overrides of the tile shape the planner would pick (0 = keep the planner's choice); for measurements.
+struct GemmTune { int mb, bn, stages; };
+
 // Bs: n_maps weight matrices [n_per_map, K] (ldb elements between rows) whose outputs are concatenated along
 // the columns of C (QKV), or gate / up for GEMM_SWIGLU (then C has n_per_map columns).
 int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int32_t K,
                          const void *const *Bs, int32_t n_maps, int32_t n_per_map, int64_t ldb,
                          int32_t mode, void *C, int64_t ldc, int32_t out_f32, float scale,
-                         __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, int32_t force_bn);
+                         __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, const GemmTune *tune);
 int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream);
 
 }  // namespace sfs

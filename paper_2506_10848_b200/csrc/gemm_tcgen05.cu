@@ -1,11 +1,17 @@
 // Dense projections of the mask predictor (QKV / O / gate-up / down / LM head): C = A * B^T with bf16
 // operands and fp32 accumulation in tensor memory.
 //
-// One CTA computes a 128 x BN output tile.  Warp 0 streams 128-byte-swizzled operand tiles into a ring of
-// shared-memory stages with TMA, warp 1 issues tcgen05.mma (one elected thread) and releases stages with
-// tcgen05.commit, warps 2-5 read the accumulator back with tcgen05.ld and run the fused epilogue
-// (scale / fp32 residual add / SwiGLU / transposed V store).  The row count may live on the device, so the
-// LM head can follow the shrinking set of masked rows without a host round trip.
+// A pair of CTAs (a cluster of two, on the two SMs of a TPC) computes a (MB x 256) x BN output tile with
+// tcgen05.mma.cta_group::2: each CTA stages its own 128 rows of every 256-row block of A and its own half of
+// the BN weight rows, so a weight tile enters the pair once and the bytes an SM pulls through its L2 port per
+// FLOP drop (the operand stream from L2, not the tensor core, bounds these shapes).  The pair walks a static
+// list of tiles (persistent kernel).  In each CTA warp 0 streams 128-byte-swizzled operand tiles into a ring of
+// shared-memory stages with TMA (completion is counted on the leader CTA's barrier), the leader's warp 1 issues
+// the MMAs and releases stages in both CTAs with a multicast tcgen05.commit, and warps 2-9 read the accumulator
+// back with tcgen05.ld and run the fused epilogue (scale / fp32 residual add / SwiGLU / transposed V store).
+// When two accumulators fit tensor memory the epilogue of a tile overlaps the next tile's main loop.  The row
+// count may live on the device, so the LM head can follow the shrinking set of masked rows without a host
+// round trip.
 #include "sfs_common.cuh"
 #include "tc05.cuh"
 #include "gemm.cuh"
@@ -50,9 +56,16 @@ int32_t make_tmap_bf16(CUtensorMap *out, const void *base, uint64_t rows, uint64
 
 namespace {
 
-constexpr int BM = 128, BK = 64;
-constexpr int kGemmThreads = 192;
+constexpr int BM = 128, BK = 64;         // rows per CTA of one 256-row MMA block; K elements per stage
+constexpr int kEpiWarps = 8;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 constexpr int A_BYTES = BM * BK * 2;
+constexpr int kMaxStages = 8;
+constexpr int kSmemBudget = 227 * 1024 - 64;      // the opt-in maximum minus the kernel's static shared memory
+// barriers: full[kMaxStages], empty[kMaxStages], acc_full[2], acc_empty[2]; then the TMEM base slot
+constexpr int kBarBytes = (2 * kMaxStages + 4) * 8 + 16;
+constexpr int kTmemCols = 512;
+constexpr int kEpiStageBytes = kEpiWarps * 32 * 128;   // one 32-row x 128-byte output unit per epilogue warp
 
 __device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
 
@@ -61,220 +74,365 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t *>(&h);
 }
 
-template <int BN, int STAGES>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+// which output columns / weight rows a tile covers
+struct TileCoord {
+    int m0;          // first output row of the pair's tile
+    int map_idx;     // which B matrix (concatenated outputs), 0 for SwiGLU
+    int n_local;     // first row of that B matrix (SwiGLU: first gate row = first up row)
+    int ncol0;       // first output column
+    int ncols;       // valid output columns of the tile (<= BN, SwiGLU: <= BN/2)
+};
+
+__device__ __forceinline__ TileCoord tile_coord(const GemmArgs &g, int tile, int m_groups)
+{
+    TileCoord t;
+    const int n_tile = tile / m_groups;
+    t.m0 = (tile - n_tile * m_groups) * (g.mb * 2 * BM);   // row groups fastest: pairs that share a weight tile run together
+    if (g.mode == GEMM_SWIGLU) {
+        const int half = g.bn >> 1;
+        t.map_idx = 0; t.n_local = n_tile * half; t.ncol0 = t.n_local; t.ncols = min(half, g.N - t.ncol0);
+    } else {
+        t.map_idx = n_tile / g.tiles_per_map;
+        t.n_local = (n_tile - t.map_idx * g.tiles_per_map) * g.bn;
+        t.ncol0 = t.map_idx * g.n_per_map + t.n_local;
+        t.ncols = min(g.bn, g.n_per_map - t.n_local);
+    }
+    return t;
+}
+
+// ---- epilogue --------------------------------------------------------------------------------------------
+// tcgen05.ld hands every lane one accumulator ROW, so storing from those registers makes each store instruction
+// touch 32 different lines.  Instead a warp parks a 32-row x 128-byte unit of output in shared memory (16-byte
+// chunks XOR-swizzled by row, so both directions are conflict-free) and writes it out as 4 rows x 128 contiguous
+// bytes per instruction.  A unit is 32 fp32 or 64 bf16 output columns.
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_add_v4_f32(float *p, uint4 v) {
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                 ::"l"(p), "f"(__uint_as_float(v.x)), "f"(__uint_as_float(v.y)), "f"(__uint_as_float(v.z)), "f"(__uint_as_float(v.w)) : "memory");
+}
+// lane = row: park 4 consecutive 16-byte chunks (chunk0 .. chunk0+3) of this lane's row
+__device__ __forceinline__ void park16(uint32_t stage, int lane, int chunk0, const uint32_t *w) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        st_shared_v4(stage + lane * 128 + (((chunk0 + c) ^ (lane & 7)) << 4), w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+}
+
+// Writes the parked unit out.  Row r of the unit is output row grow0 + r; its 128 bytes start at output column col0.
+// ELEM = bytes per output element (2 or 4); columns at or beyond `lim` and rows at or beyond M are skipped.
+// Every output element belongs to exactly one tile, so the residual add (one vector red per chunk) is deterministic.
+template <int ELEM, bool RESIDUAL>
+__device__ __forceinline__ void flush_unit(const GemmArgs &g, uint32_t stage, int lane, int grow0, int M, int col0, int lim)
+{
+    constexpr int PER = 16 / ELEM;                       // elements per 16-byte chunk
+    const int c = lane & 7, col = col0 + c * PER;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = 4 * i + (lane >> 3), grow = grow0 + r;
+        if (grow >= M || col >= lim) continue;
+        const uint4 v = ld_shared_v4(stage + r * 128 + ((c ^ (r & 7)) << 4));
+        uint8_t *dst = reinterpret_cast<uint8_t *>(g.C) + ((long long)grow * g.ldc + col) * ELEM;
+        if (col + PER <= lim) {
+            if (RESIDUAL) red_add_v4_f32(reinterpret_cast<float *>(dst), v);
+            else *reinterpret_cast<uint4 *>(dst) = v;
+        } else {                                         // ragged last chunk of the matrix: element by element
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            for (int e = 0; e < PER && col + e < lim; ++e) {
+                if (RESIDUAL) atomicAdd(reinterpret_cast<float *>(dst) + e, __uint_as_float(w[e]));
+                else if (ELEM == 4) reinterpret_cast<uint32_t *>(dst)[e] = w[e];
+                else reinterpret_cast<uint16_t *>(dst)[e] = (uint16_t)(w[e >> 1] >> ((e & 1) * 16));
+            }
+        }
+    }
+}
+
+// One warp's share of a tile's epilogue: TMEM lane quarter q (32 rows) of every 256-row block, the units of parity `par`.
+// A unit may reach past the tile's valid columns: those accumulator columns exist (inside the 256-column buffer) and
+// are never stored.
+__device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord &t, uint32_t tmem_acc, uint32_t bn_pad, uint32_t stage,
+                                              int q, int par, int lane, int rank, int M)
+{
+    const int HALF = g.bn >> 1;
+    const int lim = min(t.ncol0 + t.ncols, g.N);         // first output column this tile must not touch
+    for (int b = 0; b < g.mb; ++b) {
+        const int grow0 = t.m0 + b * 2 * BM + rank * BM + q * 32;
+        const uint32_t tbase = tmem_acc + b * bn_pad + ((uint32_t)(q * 32) << 16);
+        if (g.mode == GEMM_SWIGLU) {
+            for (int c = 64 * par; c < t.ncols; c += 128) {             // 64 outputs = 64 gate + 64 up columns
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t gt[32], up[32], o[16];
+                    tc::tmem_ld32(tbase + c + 32 * h, gt);
+                    tc::tmem_ld32(tbase + HALF + c + 32 * h, up);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        o[j] = pack_bf16(silu_f(__uint_as_float(gt[2 * j])) * __uint_as_float(up[2 * j]),
+                                         silu_f(__uint_as_float(gt[2 * j + 1])) * __uint_as_float(up[2 * j + 1]));
+                    park16(stage, lane, 4 * h, o);
+                }
+                __syncwarp();
+                flush_unit<2, false>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                __syncwarp();
+            }
+        } else if (g.vt != nullptr && t.ncol0 >= g.vt_col0) {
+            // V columns of the QKV projection go out transposed: the 32 lanes hold 32 consecutive tokens of a feature
+            const int grow = grow0 + lane;
+            for (int c = 32 * par; c < t.ncols; c += 64) {
+                uint32_t v[32];
+                tc::tmem_ld32(tbase + c, v);
+                tc::tmem_ld_wait();
+                if (grow < M) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (t.ncol0 + c + j < lim)
+                            g.vt[(long long)(t.ncol0 + c + j - g.vt_col0) * g.ldvt + grow] = __float2bfloat16_rn(__uint_as_float(v[j]) * g.scale);
+                }
+            }
+        } else if (g.mode == GEMM_RESIDUAL_F32 || g.out_f32) {
+            for (int c = 32 * par; c < t.ncols; c += 64) {              // 32 fp32 columns
+                uint32_t v[32];
+                tc::tmem_ld32(tbase + c, v);
+                tc::tmem_ld_wait();
+                if (g.mode != GEMM_RESIDUAL_F32) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * g.scale);
+                }
+                park16(stage, lane, 0, v);
+                park16(stage, lane, 4, v + 16);
+                __syncwarp();
+                if (g.mode == GEMM_RESIDUAL_F32) flush_unit<4, true>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                else flush_unit<4, false>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                __syncwarp();
+            }
+        } else {
+            for (int c = 64 * par; c < t.ncols; c += 128) {             // 64 bf16 columns
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t v[32], o[16];
+                    tc::tmem_ld32(tbase + c + 32 * h, v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) o[j] = pack_bf16(__uint_as_float(v[2 * j]) * g.scale, __uint_as_float(v[2 * j + 1]) * g.scale);
+                    park16(stage, lane, 4 * h, o);
+                }
+                __syncwarp();
+                flush_unit<2, false>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                __syncwarp();
+            }
+        }
+    }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
 {
-    constexpr int B_BYTES = BN * BK * 2;
-    constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    constexpr int HALF = BN / 2;
-
-    if (g.d_active && *g.d_active == 0) return;             // nothing left to decode: uniform early exit
+    // the exits below are uniform over the pair (same values in both CTAs), before any barrier or allocation
+    if (g.d_active && *g.d_active == 0) return;             // nothing left to decode
     const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
-    const int m_tile = blockIdx.x, n_tile = blockIdx.y;
-    const int m0 = m_tile * BM;
-    if (m0 >= M) return;                                    // uniform: before any barrier or allocation
+    const int MB = g.mb;
+    const int m_groups = (M + MB * 2 * BM - 1) / (MB * 2 * BM);
+    const int num_tiles = m_groups * g.n_col_tiles;
+    const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+    if (pair >= num_tiles) return;
+
+    const int BN = g.bn, STAGES = g.stages, HALF = BN >> 1;
+    const int STAGE_BYTES = MB * A_BYTES + HALF * BK * 2;   // per CTA: MB blocks of 128 A rows, half of the weight rows
+    const uint32_t rank = tc::cluster_ctarank();            // 0 = leader (issues the MMAs), 1 = peer
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 1);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kMaxStages + 4);
     __shared__ int s_abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_kb = (g.K + BK - 1) / BK;
     const uint32_t smem_base = tc::smem_u32(smem);
-    const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * STAGES, bar_tmem = bar_full + 16 * STAGES;
+    const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * kMaxStages;
+    const uint32_t bar_acc_full = bar_full + 16 * kMaxStages, bar_acc_empty = bar_acc_full + 16;
+    // the leader's copies of the barriers both CTAs signal
+    const uint32_t lead_full = tc::mapa(bar_full, 0), lead_acc_empty = tc::mapa(bar_acc_empty, 0);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { tc::mbar_init(bar_full + 8 * s, 1); tc::mbar_init(bar_empty + 8 * s, 1); }
-        tc::mbar_init(bar_tmem, 1);
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(bar_acc_full + 8 * b, 1); tc::mbar_init(bar_acc_empty + 8 * b, 2 * kEpiWarps); }
         s_abort = 0;
         tc::mbar_init_fence();
     }
-    if (warp == 1) { tc::tmem_alloc(tc::smem_u32(tmem_slot), BN); tc::tmem_relinquish(); }
+    __syncwarp();
+    if (warp == 1) { tc::tmem_alloc_2cta(tc::smem_u32(tmem_slot), kTmemCols); tc::tmem_relinquish_2cta(); }
     tc::tc_fence_before();
-    __syncthreads();
+    tc::cluster_sync();                                     // barriers of both CTAs are initialised, TMEM is allocated
     tc::tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
-
-    // which B rows feed this tile
+    const uint32_t bn_pad = (uint32_t)((BN + 31) & ~31);
+    const uint32_t n_bufs = (uint32_t)g.acc_bufs, buf_stride = 256;     // two buffers only when MB * bn_pad <= 256
     const bool swiglu = (g.mode == GEMM_SWIGLU);
-    const int map_idx = swiglu ? 0 : (n_tile / g.tiles_per_map);
-    const int n_local = swiglu ? n_tile * HALF : (n_tile % g.tiles_per_map) * BN;
 
+    // The producer and MMA loops are run by all 32 lanes of their warp with warp-uniform operands; one elected lane
+    // issues each asynchronous instruction.  (Issued from a single-lane branch, every tcgen05.mma cost the thread
+    // about 90 cycles and an already-complete mbarrier wait about 200: the loop, not the tensor core, set the pace.)
+    // The readiness of the next stage is polled (without blocking) before the current stage's instructions are
+    // issued, so the latency of that poll overlaps the issue.
     if (warp == 0) {
-        if (lane == 0) {
-            // ---------------- TMA producer
-            tc::tma_prefetch_desc(&tmA);
-            const CUtensorMap *mb0 = swiglu ? &tmB0 : (map_idx == 0 ? &tmB0 : (map_idx == 1 ? &tmB1 : &tmB2));
-            const CUtensorMap *mb1 = swiglu ? &tmB1 : mb0;
-            const int row1 = swiglu ? n_local : n_local + HALF;
-            int issued = 0;
-            for (int kb = 0; kb < num_kb; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-                if (!tc::mbar_wait(bar_empty + 8 * s, ph ^ 1u, &s_abort)) break;
-                const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-                tc::mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
-                tc::tma_load_2d(sa, &tmA, kb * BK, m0, bar_full + 8 * s);
-                tc::tma_load_2d(sb, mb0, kb * BK, n_local, bar_full + 8 * s);
-                tc::tma_load_2d(sb + HALF * BK * 2, mb1, kb * BK, row1, bar_full + 8 * s);
-                issued = kb + 1;
+        // ---------------- TMA producer (both CTAs; completion bytes are counted on the leader's barrier)
+        if (lane == 0) { tc::tma_prefetch_desc(&tmA); tc::tma_prefetch_desc(&tmB0); }
+        uint32_t it = 0;
+        bool ok = true;
+        bool ready = tc::mbar_test(bar_empty, 1u);
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
+            const TileCoord t = tile_coord(g, tile, m_groups);
+            // leader: first half of the weight rows (SwiGLU: the gate rows); peer: second half (the up rows)
+            const CUtensorMap *mb = swiglu ? (rank == 0 ? &tmB0 : &tmB1)
+                                           : (t.map_idx == 0 ? &tmB0 : (t.map_idx == 1 ? &tmB1 : &tmB2));
+            const int brow = swiglu ? t.n_local : t.n_local + (int)rank * HALF;
+            const int arow = t.m0 + (int)rank * BM;
+            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const uint32_t s = it % (uint32_t)STAGES, ph = (it / (uint32_t)STAGES) & 1u;
+                if (!ready) ready = tc::mbar_wait(bar_empty + 8 * s, ph ^ 1u, &s_abort);
+                ok = __all_sync(0xffffffffu, ready);
+                if (!ok) break;
+                const uint32_t nx = it + 1u, ns = nx % (uint32_t)STAGES, nph = (nx / (uint32_t)STAGES) & 1u;
+                ready = tc::mbar_test(bar_empty + 8 * ns, nph ^ 1u);
+                const uint32_t sa = smem_base + s * STAGE_BYTES;
+                if (rank == 0) tc::mbar_expect_tx_elect(bar_full + 8 * s, 2u * (uint32_t)STAGE_BYTES);
+                tc::tma_load_2d_2cta_elect(sa, &tmA, kb * BK, arow, lead_full + 8 * s);
+                if (MB == 2) tc::tma_load_2d_2cta_elect(sa + A_BYTES, &tmA, kb * BK, arow + 2 * BM, lead_full + 8 * s);
+                tc::tma_load_2d_2cta_elect(sa + MB * A_BYTES, mb, kb * BK, brow, lead_full + 8 * s);
             }
-            if (s_abort) {
-                // give copies already in flight a bounded chance to land before the CTA retires
-                for (int kb = max(0, issued - STAGES); kb < issued; ++kb) {
-                    const uint32_t bar = bar_full + 8 * (kb % STAGES), ph = (uint32_t)(kb / STAGES) & 1u;
-                    for (int i = 0; i < (1 << 16) && !tc::mbar_try(bar, ph); ++i) {}
-                }
+        }
+        if (s_abort && rank == 0 && lane == 0) {
+            // give copies already in flight (both CTAs') a bounded chance to land before the pair retires
+            const uint32_t first = it > (uint32_t)STAGES ? it - (uint32_t)STAGES : 0u;
+            for (uint32_t j = first; j < it; ++j) {
+                const uint32_t bar = bar_full + 8 * (j % (uint32_t)STAGES), ph = (j / (uint32_t)STAGES) & 1u;
+                for (int i = 0; i < (1 << 16) && !tc::mbar_try(bar, ph); ++i) {}
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
-            constexpr uint32_t idesc = tc::idesc_bf16_f32(BM, BN);
+        if (rank == 0) {
+            // ---------------- MMA issuer (leader CTA only)
+            const uint32_t idesc = tc::idesc_bf16_f32(2 * BM, BN);
+            uint32_t it = 0, lt = 0;
             bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; ++kb) {
-                const int s = kb % STAGES;
-                const uint32_t ph = (uint32_t)(kb / STAGES) & 1u;
-                ok = tc::mbar_wait(bar_full + 8 * s, ph, &s_abort);
+            bool ready = tc::mbar_test(bar_full, 0u);
+            for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++lt) {
+                const uint32_t buf = lt % n_bufs, use = lt / n_bufs;
+                // both CTAs' epilogues have drained this accumulator buffer
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(bar_acc_empty + 8 * buf, (use & 1u) ^ 1u, &s_abort));
                 if (!ok) break;
                 tc::tc_fence_after();
-                const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-                const uint64_t da = tc::smem_desc_sw128(sa), db = tc::smem_desc_sw128(sb);
+                const uint32_t d_tmem = tmem_base + buf * buf_stride;
+                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                    const uint32_t s = it % (uint32_t)STAGES, ph = (it / (uint32_t)STAGES) & 1u;
+                    if (!ready) ready = tc::mbar_wait(bar_full + 8 * s, ph, &s_abort);
+                    ok = __all_sync(0xffffffffu, ready);
+                    if (!ok) break;
+                    tc::tc_fence_after();
+                    const uint32_t nx = it + 1u, ns = nx % (uint32_t)STAGES, nph = (nx / (uint32_t)STAGES) & 1u;
+                    ready = tc::mbar_test(bar_full + 8 * ns, nph);
+                    const uint32_t sa = smem_base + s * STAGE_BYTES;
+                    const uint64_t da = tc::smem_desc_sw128(sa), db = tc::smem_desc_sw128(sa + MB * A_BYTES);
+                    const uint32_t acc = kb != 0 ? 1u : 0u;
+                    tc::mma_bf16_2cta_elect(d_tmem, da, db, idesc, acc);
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; ++kk)
-                    tc::mma_bf16(tmem_base, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, (kb | kk) != 0 ? 1u : 0u);
-                tc::mma_commit(bar_empty + 8 * s);           // frees the stage once these MMAs have read it
+                    for (int kk = 1; kk < BK / 16; ++kk) tc::mma_bf16_2cta_elect(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, 1u);
+                    if (MB == 2) {
+                        const uint64_t da1 = tc::smem_desc_sw128(sa + A_BYTES);
+                        tc::mma_bf16_2cta_elect(d_tmem + bn_pad, da1, db, idesc, acc);
+#pragma unroll
+                        for (int kk = 1; kk < BK / 16; ++kk) tc::mma_bf16_2cta_elect(d_tmem + bn_pad, da1 + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, 1u);
+                    }
+                    tc::mma_commit_2cta_elect(bar_empty + 8 * s);     // frees the stage in both CTAs once these MMAs have read it
+                }
+                tc::mma_commit_2cta_elect(bar_acc_full + 8 * buf);    // accumulator complete (or abandoned), both CTAs
             }
-            tc::mma_commit(bar_tmem);                        // accumulator complete (or abandoned)
         }
     } else {
-        // ---------------- epilogue: 4 warps, one TMEM lane quarter each
-        const int q = warp & 3;
-        const int row = q * 32 + lane;
-        const int grow = m0 + row;
-        const bool row_ok = grow < M;
-        const bool ok = tc::mbar_wait(bar_tmem, 0, &s_abort) && !s_abort;
-        tc::tc_fence_after();
-        const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16);
-        if (ok) {
-            if (swiglu) {
-                __nv_bfloat16 *C = reinterpret_cast<__nv_bfloat16 *>(g.C);
-                for (int c = 0; c < HALF / 32; ++c) {
-                    uint32_t gt[32], up[32];
-                    tc::tmem_ld32(tbase + c * 32, gt);
-                    tc::tmem_ld32(tbase + HALF + c * 32, up);
-                    tc::tmem_ld_wait();
-                    const int col0 = n_local + c * 32;
-                    if (row_ok) {
-                        __nv_bfloat16 *dst = C + (long long)grow * g.ldc + col0;
-                        if (col0 + 32 <= g.N) {
-                            uint32_t o[16];
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const float a = silu_f(__uint_as_float(gt[2 * j])) * __uint_as_float(up[2 * j]);
-                                const float b = silu_f(__uint_as_float(gt[2 * j + 1])) * __uint_as_float(up[2 * j + 1]);
-                                o[j] = pack_bf16(a, b);
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                reinterpret_cast<uint4 *>(dst)[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-                        } else {
-                            _Pragma("unroll")
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < g.N) dst[j] = __float2bfloat16_rn(silu_f(__uint_as_float(gt[j])) * __uint_as_float(up[j]));
-                        }
-                    }
-                }
-            } else {
-                const int ncol0 = n_tile * BN;
-                const bool to_vt = (g.vt != nullptr) && (ncol0 >= g.vt_col0);
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t v[32];
-                    tc::tmem_ld32(tbase + c * 32, v);
-                    tc::tmem_ld_wait();
-                    const int col0 = ncol0 + c * 32;
-                    if (!row_ok || col0 >= g.N) continue;
-                    const bool full = col0 + 32 <= g.N;
-                    if (g.mode == GEMM_RESIDUAL_F32) {
-                        float *dst = reinterpret_cast<float *>(g.C) + (long long)grow * g.ldc + col0;
-                        if (full) {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) {
-                                float4 x = reinterpret_cast<float4 *>(dst)[j];
-                                x.x += __uint_as_float(v[4 * j]);     x.y += __uint_as_float(v[4 * j + 1]);
-                                x.z += __uint_as_float(v[4 * j + 2]); x.w += __uint_as_float(v[4 * j + 3]);
-                                reinterpret_cast<float4 *>(dst)[j] = x;
-                            }
-                        } else {
-                            _Pragma("unroll")
-                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] += __uint_as_float(v[j]);
-                        }
-                    } else if (to_vt) {
-                        // transposed store: 32 lanes hold 32 consecutive tokens of one feature column
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < g.N)
-                                g.vt[(long long)(col0 + j - g.vt_col0) * g.ldvt + grow] = __float2bfloat16_rn(__uint_as_float(v[j]) * g.scale);
-                    } else if (g.out_f32) {
-                        float *dst = reinterpret_cast<float *>(g.C) + (long long)grow * g.ldc + col0;
-                        if (full) {
-#pragma unroll
-                            for (int j = 0; j < 8; ++j)
-                                reinterpret_cast<float4 *>(dst)[j] = make_float4(__uint_as_float(v[4 * j]) * g.scale, __uint_as_float(v[4 * j + 1]) * g.scale,
-                                                                                 __uint_as_float(v[4 * j + 2]) * g.scale, __uint_as_float(v[4 * j + 3]) * g.scale);
-                        } else {
-                            _Pragma("unroll")
-                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(v[j]) * g.scale;
-                        }
-                    } else {
-                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(g.C) + (long long)grow * g.ldc + col0;
-                        if (full) {
-                            uint32_t o[16];
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) o[j] = pack_bf16(__uint_as_float(v[2 * j]) * g.scale, __uint_as_float(v[2 * j + 1]) * g.scale);
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                reinterpret_cast<uint4 *>(dst)[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
-                        } else {
-                            _Pragma("unroll")
-                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]) * g.scale);
-                        }
-                    }
-                }
-            }
+        // ---------------- epilogue: 8 warps; warp w reads TMEM lanes 32*(w%4).., the column units of parity (w-2)/4
+        const int q = warp & 3, par = (warp - 2) >> 2;
+        const uint32_t stage = smem_base + STAGES * STAGE_BYTES + kBarBytes + (uint32_t)(warp - 2) * (32 * 128);
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int tile = pair; tile < num_tiles && ok; tile += num_pairs, ++lt) {
+            const TileCoord t = tile_coord(g, tile, m_groups);
+            const uint32_t buf = lt % n_bufs, use = lt / n_bufs;
+            ok = tc::mbar_wait(bar_acc_full + 8 * buf, use & 1u, &s_abort) && !s_abort;
+            if (!ok) break;
+            tc::tc_fence_after();
+            epilogue_tile(g, t, tmem_base + buf * buf_stride, bn_pad, stage, q, par, lane, (int)rank, M);
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive_cluster(lead_acc_empty + 8 * buf);
         }
     }
 
-    // ---------------- teardown
+    // ---------------- teardown: no CTA of the pair leaves while the other may still signal its barriers
+    __syncwarp();                                           // the diverged roles rejoin their warps
     tc::tc_fence_before();
-    __syncthreads();
-    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, BN); }
+    tc::cluster_sync();
+    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc_2cta(tmem_base, kTmemCols); }
     if (threadIdx.x == 0 && s_abort && g.err) atomicExch(g.err, SFS_ERR_TIMEOUT);
 }
 
-template <int BN, int STAGES>
-int32_t launch_cfg(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream)
+int num_sms()
 {
-    constexpr size_t smem = (size_t)STAGES * (A_BYTES + BN * BK * 2) + (2 * STAGES + 1) * 8 + 16 + 1024;
-    static bool configured = false;
-    if (!configured) {
-        SFS_CUDA(cudaFuncSetAttribute(gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
     }
-    GemmArgs g = p.args;
-    g.d_m = d_m; g.err = err; g.d_active = d_active;
-    const int cols_per_tile = (g.mode == GEMM_SWIGLU) ? BN / 2 : BN;
-    int n_tiles;
-    if (g.mode == GEMM_SWIGLU || p.n_maps == 1) { n_tiles = (g.N + cols_per_tile - 1) / cols_per_tile; g.tiles_per_map = 0x3FFFFFFF; }
-    else { g.tiles_per_map = p.n_per_map / BN; n_tiles = g.tiles_per_map * p.n_maps; }
-    dim3 grid((unsigned)((g.M + BM - 1) / BM), (unsigned)n_tiles, 1);
-    gemm_kernel<BN, STAGES><<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
-    SFS_LAUNCH_CHECK();
-    return SFS_OK;
+    return n;
+}
+
+// column tiles of a problem at tile width bn
+int col_tiles(int mode, int n_maps, int n_per_map, int bn)
+{
+    if (mode == GEMM_SWIGLU) return (n_per_map + bn / 2 - 1) / (bn / 2);
+    return n_maps * ((n_per_map + bn - 1) / bn);
+}
+
+int stages_for(int mb, int bn)
+{
+    const int stage_bytes = mb * A_BYTES + (bn / 2) * BK * 2;
+    const int s = (kSmemBudget - 1024 - kBarBytes - kEpiStageBytes) / stage_bytes;
+    return s > kMaxStages ? kMaxStages : s;
+}
+
+// Tile shape (MB blocks of 256 rows, width bn): the candidate with the smallest modelled time
+//   waves x (k-blocks x max(MMA clocks, operand-stream clocks) + exposed epilogue clocks)
+// per pair of SMs.  Per k-block and CTA the tensor core needs MB*bn*2 clocks (8192 FLOP/clk/SM); the operand
+// stream is (MB*128 + bn/2) rows x 128 B at the ~40 B/clk an SM sustains from L2 when every SM streams (measured),
+// with a floor for the per-k-block handshakes.  The epilogue is hidden behind the next tile when two accumulators
+// fit tensor memory, except for the last tile of a pair.
+void pick_tile(int M, int K, int mode, int n_maps, int n_per_map, int pairs, int *mb_out, int *bn_out)
+{
+    const int step = (mode == GEMM_SWIGLU) ? 32 : 16;
+    const long long num_kb = (K + BK - 1) / BK;
+    long long best_cost = -1;
+    for (int mb = (M > 2 * BM ? 2 : 1); mb >= 1; --mb) {
+        const int m_groups = (M + mb * 2 * BM - 1) / (mb * 2 * BM);
+        for (int bn = 256; bn >= 32; bn -= step) {
+            const long long tiles = (long long)m_groups * col_tiles(mode, n_maps, n_per_map, bn);
+            const long long waves = (tiles + pairs - 1) / pairs;
+            const long long mma = (long long)mb * bn * 2, load = (long long)(mb * BM + bn / 2) * 128 / 40;
+            long long kb_clk = mma > load ? mma : load;
+            if (kb_clk < 450) kb_clk = 450;
+            const long long epi = (long long)mb * bn * 16 + 3000;
+            const bool hidden = mb * ((bn + 31) & ~31) <= 256;
+            const long long cost = waves * num_kb * kb_clk + (hidden ? 1 : waves) * epi;
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; *mb_out = mb; *bn_out = bn; }
+        }
+    }
 }
 
 }  // namespace
@@ -282,7 +440,7 @@ int32_t launch_cfg(const GemmPlan &p, const int32_t *d_m, const int32_t *d_activ
 int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int32_t K,
                          const void *const *Bs, int32_t n_maps, int32_t n_per_map, int64_t ldb,
                          int32_t mode, void *C, int64_t ldc, int32_t out_f32, float scale,
-                         __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, int32_t force_bn)
+                         __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, const GemmTune *tune)
 {
     SFS_REQUIRE(M >= 1 && K >= 1 && n_per_map >= 1 && n_maps >= 1 && n_maps <= 3, SFS_ERR_INVALID_ARG, "gemm: bad sizes");
     SFS_REQUIRE((K % 8) == 0 && (lda % 8) == 0 && (ldb % 8) == 0, SFS_ERR_INVALID_ARG, "gemm: K, lda, ldb must be multiples of 8");
@@ -290,14 +448,12 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     memset(p, 0, sizeof(*p));
     const int N = (mode == GEMM_SWIGLU) ? n_per_map : n_per_map * n_maps;
     SFS_REQUIRE(aligned_to(C, 16) && (ldc % 8) == 0, SFS_ERR_INVALID_ARG, "gemm: C must be 16-byte aligned, ldc a multiple of 8");
-    // tile width: wide tiles when they still fill the machine, else narrow ones
-    const int m_tiles = (M + BM - 1) / BM;
-    const int cols256 = (mode == GEMM_SWIGLU) ? 128 : 256;
-    int bn = ((long long)m_tiles * ((N + cols256 - 1) / cols256) >= 148) ? 256 : 128;
-    if (n_maps > 1 && mode != GEMM_SWIGLU && (n_per_map % 256) != 0) bn = 128;
-    if (force_bn == 128 || force_bn == 256) bn = force_bn;
-    SFS_REQUIRE(n_maps == 1 || mode == GEMM_SWIGLU || (n_per_map % bn) == 0, SFS_ERR_UNSUPPORTED,
-                "gemm: concatenated outputs need a width that is a multiple of %d (got %d)", bn, n_per_map);
+    int mb = 1, bn = 256;
+    pick_tile(M, K, mode, n_maps, n_per_map, num_sms() / 2, &mb, &bn);
+    if (tune) {                                              // measurement overrides; invalid values are ignored
+        if (tune->mb == 1 || tune->mb == 2) mb = tune->mb;
+        if (tune->bn >= 32 && tune->bn <= 256 && (tune->bn % ((mode == GEMM_SWIGLU) ? 32 : 16)) == 0) bn = tune->bn;
+    }
     p->bn = bn; p->n_maps = n_maps; p->n_per_map = n_per_map;
     int32_t rc = make_tmap_bf16(&p->tmA, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM);
     if (rc != SFS_OK) return rc;
@@ -309,13 +465,34 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     GemmArgs &g = p->args;
     g.M = M; g.N = N; g.K = K; g.mode = mode; g.out_f32 = out_f32; g.scale = scale;
     g.C = C; g.ldc = ldc; g.vt = vt; g.ldvt = ldvt; g.vt_col0 = vt_col0;
+    g.bn = bn; g.mb = mb; g.n_per_map = n_per_map;
+    g.tiles_per_map = (mode == GEMM_SWIGLU) ? 0x3FFFFFFF : (n_per_map + bn - 1) / bn;
+    g.n_col_tiles = col_tiles(mode, n_maps, n_per_map, bn);
+    g.stages = stages_for(mb, bn);
+    if (tune && tune->stages >= 1 && tune->stages <= g.stages) g.stages = tune->stages;
+    g.acc_bufs = (mb * ((bn + 31) & ~31) <= 256) ? 2 : 1;
     return SFS_OK;
 }
 
 int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
-    if (p.bn == 256) return launch_cfg<256, 4>(p, d_m, d_active, err, stream);
-    return launch_cfg<128, 6>(p, d_m, d_active, err, stream);
+    // always ask for more than half of an SM's shared memory: one CTA per SM, so the allocation of all 512
+    // tensor-memory columns can never wait for a co-resident CTA
+    static bool configured = false;
+    if (!configured) {
+        SFS_CUDA(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        configured = true;
+    }
+    GemmArgs g = p.args;
+    g.d_m = d_m; g.err = err; g.d_active = d_active;
+    size_t smem = (size_t)g.stages * (g.mb * A_BYTES + (g.bn / 2) * BK * 2) + kBarBytes + kEpiStageBytes + 1024;
+    if (smem < 120 * 1024) smem = 120 * 1024;
+    const long long tiles = (long long)((g.M + g.mb * 2 * BM - 1) / (g.mb * 2 * BM)) * g.n_col_tiles;
+    const int pairs = num_sms() / 2;
+    dim3 grid((unsigned)(2 * (tiles < pairs ? tiles : pairs)), 1, 1);
+    gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
 }
 
 }  // namespace sfs
