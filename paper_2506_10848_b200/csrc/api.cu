@@ -12,6 +12,7 @@
 namespace sfs {
 
 static thread_local char g_err[512] = "";
+static constexpr int kMaxSplits = 6;           // slabs of the split-K workspace of the residual projections
 
 void set_error(const char *fmt, ...)
 {
@@ -87,12 +88,14 @@ static int32_t session_plan(sfs_session *s, int32_t B, int32_t S)
         const void *wo[1] = {m->wo[l]};
         rc = gemm_plan_create(&lp.o, s->attn, d, T, d, wo, 1, d, d, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
+        if ((rc = gemm_plan_enable_split(&lp.o, s->partial, kMaxSplits, nullptr)) != SFS_OK) return rc;
         const void *gu[2] = {m->w_gate[l], m->w_up[l]};
         rc = gemm_plan_create(&lp.gate_up, s->h, d, T, d, gu, 2, ff, d, GEMM_SWIGLU, s->hid, ff, 0, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
         const void *wd[1] = {m->w_down[l]};
         rc = gemm_plan_create(&lp.down, s->hid, ff, T, ff, wd, 1, d, ff, GEMM_RESIDUAL_F32, s->x, d, 1, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
+        if ((rc = gemm_plan_enable_split(&lp.down, s->partial, kMaxSplits, nullptr)) != SFS_OK) return rc;
     }
     rc = attn_plan_create(&s->attn_plan, s->qk, 2 * d, s->vt, T, s->attn, d, B, S, c.n_heads, c.head_dim);
     if (rc != SFS_OK) return rc;
@@ -125,17 +128,23 @@ static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int3
     SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
     int32_t rc;
     if ((rc = timed_launch(s, SFS_K_EMBED, st, [&] { return launch_embed(d_tokens, m->tok_emb, s->x, T, d, c.vocab, st); })) != SFS_OK) return rc;
+    // A split-K projection leaves its partial products in s->partial; the next RMSNorm folds them into x.
+    const long long pstride = (long long)T * d;
+    int pending = 0;
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerPlans &lp = s->layer_plans[l];
-        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, m->attn_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, pending, pstride, m->attn_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(lp.qkv, nullptr, d_active, err, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch(s->attn_plan, d_active, err, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(lp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, m->mlp_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
+        pending = lp.o.args.splits > 1 ? lp.o.args.splits : 0;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, pending, pstride, m->mlp_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(lp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(lp.down, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+        pending = lp.down.args.splits > 1 ? lp.down.args.splits : 0;
     }
+    s->pending_partials = pending;                           // for the final RMSNorm of the caller
     return SFS_OK;
 }
 
@@ -276,6 +285,7 @@ int32_t sfs_session_create(sfs_model *m, int32_t max_batch, int32_t max_seq, sfs
     if (rc != SFS_OK) return fail(rc);
     if ((rc = dev_alloc(s, &s->x, T * d, false)) != SFS_OK) return fail(rc);
     if ((rc = dev_alloc(s, &s->h, T * d, false)) != SFS_OK) return fail(rc);
+    if ((rc = dev_alloc(s, &s->partial, (size_t)kMaxSplits * T * d, false)) != SFS_OK) return fail(rc);
     if ((rc = dev_alloc(s, &s->qk, T * 2 * d, false)) != SFS_OK) return fail(rc);
     if ((rc = dev_alloc(s, &s->vt, T * d, false)) != SFS_OK) return fail(rc);
     if ((rc = dev_alloc(s, &s->attn, T * d, false)) != SFS_OK) return fail(rc);
@@ -320,7 +330,7 @@ int32_t sfs_forward(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t 
     int32_t rc = session_plan(s, B, S);
     if (rc != SFS_OK) return rc;
     if ((rc = run_body(s, d_tokens, B, S, nullptr, st)) != SFS_OK) return rc;
-    if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
+    if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, s->pending_partials, (long long)B * S * c.d_model, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
     GemmPlan lm;
     const void *lmw[1] = {s->model->lm_head};
     rc = gemm_plan_create(&lm, s->hfin, c.d_model, max_rows, c.d_model, lmw, 1, c.vocab, c.d_model, GEMM_STORE, d_logits, c.vocab,
@@ -433,7 +443,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         const int32_t *d_active = s->ctrl + 2;
         const int32_t *rows = s->rows[cur], *n_rows = s->ctrl + cur;
         if ((rc = run_body(s, s->tokens, B, S, d_active, st)) != SFS_OK) return rc;
-        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, s->pending_partials, (long long)B * S * c.d_model, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(s->lm_plan, n_rows, d_active, err, st); })) != SFS_OK) return rc;
         if (d_logits_dump) {
             SFS_CUDA(cudaMemcpyAsync(d_logits_dump, s->logits, (size_t)B * L * c.vocab * 2, cudaMemcpyDeviceToDevice, st));

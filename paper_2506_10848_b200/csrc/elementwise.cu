@@ -25,20 +25,36 @@ __global__ void embed_kernel(const int32_t *__restrict__ tokens, const __nv_bflo
     }
 }
 
-// h[r, :] = bf16( x[src(r), :] * rsqrt(mean(x^2) + eps) * g ),  src(r) = rows ? rows[r] : r
-constexpr int kNormThreads = 128;
+// h[r, :] = bf16( y * rsqrt(mean(y^2) + eps) * g ),  y = x[src(r), :] + sum_s partial[s][src(r), :],  src(r) = rows ? rows[r] : r.
+// The partial products of a split-K projection are added in slab order (the sum does not depend on which CTA of the
+// projection finished first); without a row list y is written back to x, so the residual stream is complete again.
+// A thread keeps its part of the row in registers between the two passes (rows of up to kNormThreads * 16 elements).
+constexpr int kNormThreads = 256;
+constexpr int kNormRegChunks = 4;                          // float4 chunks a thread keeps
 __global__ void __launch_bounds__(kNormThreads)
-rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
+rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ partial, int n_partial, long long partial_stride,
+               const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
                const int32_t *__restrict__ rows, const int32_t *__restrict__ n_rows_ptr, int max_rows, int d, float eps)
 {
     const int n_rows = n_rows_ptr ? min(*n_rows_ptr, max_rows) : max_rows;
     __shared__ float s_part[kNormThreads / 32];
+    const int chunks = d / 4;
     for (int r = blockIdx.x; r < n_rows; r += gridDim.x) {
         const long long src = rows ? rows[r] : r;
-        const float4 *xr = reinterpret_cast<const float4 *>(x + src * d);
+        float4 *xr = reinterpret_cast<float4 *>(x + src * d);
+        const float4 *pr = reinterpret_cast<const float4 *>(partial + src * d);
+        const long long pstride4 = partial_stride / 4;
+        float4 keep[kNormRegChunks];
         float ss = 0.f;
-        for (int c = threadIdx.x; c < d / 4; c += kNormThreads) {
-            const float4 v = xr[c];
+        int k = 0;
+        for (int c = threadIdx.x; c < chunks; c += kNormThreads, ++k) {
+            float4 v = xr[c];
+            for (int s = 0; s < n_partial; ++s) {
+                const float4 p = pr[(long long)s * pstride4 + c];
+                v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+            }
+            if (n_partial > 0 && rows == nullptr) xr[c] = v;
+            if (k < kNormRegChunks) keep[k] = v;
             ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         }
         ss = warp_sum(ss);
@@ -50,8 +66,18 @@ rmsnorm_kernel(const float *__restrict__ x, const __nv_bfloat16 *__restrict__ ga
         const float inv = rsqrtf(tot / (float)d + eps);
         const uint2 *gp = reinterpret_cast<const uint2 *>(gain);
         uint2 *hp = reinterpret_cast<uint2 *>(h + (long long)r * d);
-        for (int c = threadIdx.x; c < d / 4; c += kNormThreads) {
-            const float4 v = xr[c];
+        k = 0;
+        for (int c = threadIdx.x; c < chunks; c += kNormThreads, ++k) {
+            float4 v;
+            if (k < kNormRegChunks) v = keep[k];
+            else {                                           // long rows: rebuild the value the first pass saw
+                v = xr[c];
+                if (rows != nullptr)
+                    for (int s = 0; s < n_partial; ++s) {
+                        const float4 p = pr[(long long)s * pstride4 + c];
+                        v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+                    }
+            }
             const uint2 g = gp[c];
             __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * inv * bf16_bits_to_f32(g.x & 0xFFFFu), v.y * inv * bf16_bits_to_f32(g.x >> 16));
             __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * inv * bf16_bits_to_f32(g.y & 0xFFFFu), v.w * inv * bf16_bits_to_f32(g.y >> 16));
@@ -116,12 +142,13 @@ int32_t launch_embed(const int32_t *tokens, const void *emb, float *x, int T, in
     return SFS_OK;
 }
 
-int32_t launch_rmsnorm(const float *x, const void *gain, void *h, const int32_t *rows, const int32_t *n_rows,
-                       int max_rows, int d, float eps, cudaStream_t s)
+int32_t launch_rmsnorm(float *x, const float *partial, int n_partial, long long partial_stride, const void *gain, void *h,
+                       const int32_t *rows, const int32_t *n_rows, int max_rows, int d, float eps, cudaStream_t s)
 {
     if (max_rows <= 0) return SFS_OK;
     const int grid = max_rows < 148 * 16 ? max_rows : 148 * 16;
-    rmsnorm_kernel<<<grid, kNormThreads, 0, s>>>(x, reinterpret_cast<const __nv_bfloat16 *>(gain),
+    if (partial == nullptr) n_partial = 0;
+    rmsnorm_kernel<<<grid, kNormThreads, 0, s>>>(x, partial ? partial : x, n_partial, partial_stride, reinterpret_cast<const __nv_bfloat16 *>(gain),
                                                  reinterpret_cast<__nv_bfloat16 *>(h), rows, n_rows, max_rows, d, eps);
     SFS_LAUNCH_CHECK();
     return SFS_OK;

@@ -24,6 +24,8 @@ struct GemmArgs {
     int bn, stages;          // tile width (multiple of 16, <= 256) and depth of the shared-memory ring
     int mb;                  // 256-row blocks per tile (1 or 2)
     int n_col_tiles;         // column tiles over all B matrices
+    int splits, kb_per_split;        // split-K: the k-blocks are cut into `splits` ranges, range s writes slab s of C
+    long long split_stride;          // elements between slabs
     int acc_bufs;            // accumulator buffers in tensor memory (2 when they fit: epilogue overlaps the next tile)
     int32_t *err;            // device status word, set to SFS_ERR_TIMEOUT if a bounded wait gives up
     const int32_t *d_active; // optional: the kernel does nothing when *d_active == 0
@@ -33,10 +35,11 @@ struct GemmPlan {
     CUtensorMap tmA, tmB[3];
     GemmArgs args;
     int bn, n_maps, n_per_map;
+    const void *A, *Bs[3]; long long lda, ldb;       // kept so that the plan can be rebuilt at another tile shape
 };
 
 // Optional overrides of the tile shape the planner would pick (0 = keep the planner's choice); for measurements.
-struct GemmTune { int mb, bn, stages; };
+struct GemmTune { int mb, bn, stages, splits; };
 
 // Bs: n_maps weight matrices [n_per_map, K] (ldb elements between rows) whose outputs are concatenated along
 // the columns of C (QKV), or gate / up for GEMM_SWIGLU (then C has n_per_map columns).
@@ -44,6 +47,11 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
                          const void *const *Bs, int32_t n_maps, int32_t n_per_map, int64_t ldb,
                          int32_t mode, void *C, int64_t ldc, int32_t out_f32, float scale,
                          __nv_bfloat16 *vt, int64_t ldvt, int32_t vt_col0, const GemmTune *tune);
+// Split-K for the residual projections (mode GEMM_RESIDUAL_F32): when `ws` is given and the planner finds that cutting
+// K fills the machine better, the plan writes `args.splits` fp32 partial products to the slabs ws + s * M * ldc (plain
+// stores, C itself is not touched) and the consumer of the residual stream adds them in slab order (launch_rmsnorm does),
+// so the sum does not depend on which CTA finishes first.  ws must hold max_splits * M * ldc floats.
+int32_t gemm_plan_enable_split(GemmPlan *p, float *ws, int32_t max_splits, const GemmTune *tune);
 int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_active, int32_t *err, cudaStream_t stream);
 
 }  // namespace sfs

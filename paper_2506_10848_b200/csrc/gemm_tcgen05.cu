@@ -76,6 +76,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 
 // which output columns / weight rows a tile covers
 struct TileCoord {
+    int split;       // which range of k-blocks (split-K), 0 when K is not split
     int m0;          // first output row of the pair's tile
     int map_idx;     // which B matrix (concatenated outputs), 0 for SwiGLU
     int n_local;     // first row of that B matrix (SwiGLU: first gate row = first up row)
@@ -86,8 +87,10 @@ struct TileCoord {
 __device__ __forceinline__ TileCoord tile_coord(const GemmArgs &g, int tile, int m_groups)
 {
     TileCoord t;
-    const int n_tile = tile / m_groups;
-    t.m0 = (tile - n_tile * m_groups) * (g.mb * 2 * BM);   // row groups fastest: pairs that share a weight tile run together
+    const int rest = tile / m_groups;
+    t.m0 = (tile - rest * m_groups) * (g.mb * 2 * BM);     // row groups fastest: pairs that share a weight tile run together
+    const int n_tile = rest / g.splits;
+    t.split = rest - n_tile * g.splits;
     if (g.mode == GEMM_SWIGLU) {
         const int half = g.bn >> 1;
         t.map_idx = 0; t.n_local = n_tile * half; t.ncol0 = t.n_local; t.ncols = min(half, g.N - t.ncol0);
@@ -128,7 +131,7 @@ __device__ __forceinline__ void park16(uint32_t stage, int lane, int chunk0, con
 // ELEM = bytes per output element (2 or 4); columns at or beyond `lim` and rows at or beyond M are skipped.
 // Every output element belongs to exactly one tile, so the residual add (one vector red per chunk) is deterministic.
 template <int ELEM, bool RESIDUAL>
-__device__ __forceinline__ void flush_unit(const GemmArgs &g, uint32_t stage, int lane, int grow0, int M, int col0, int lim)
+__device__ __forceinline__ void flush_unit(const GemmArgs &g, long long slab, uint32_t stage, int lane, int grow0, int M, int col0, int lim)
 {
     constexpr int PER = 16 / ELEM;                       // elements per 16-byte chunk
     const int c = lane & 7, col = col0 + c * PER;
@@ -137,7 +140,7 @@ __device__ __forceinline__ void flush_unit(const GemmArgs &g, uint32_t stage, in
         const int r = 4 * i + (lane >> 3), grow = grow0 + r;
         if (grow >= M || col >= lim) continue;
         const uint4 v = ld_shared_v4(stage + r * 128 + ((c ^ (r & 7)) << 4));
-        uint8_t *dst = reinterpret_cast<uint8_t *>(g.C) + ((long long)grow * g.ldc + col) * ELEM;
+        uint8_t *dst = reinterpret_cast<uint8_t *>(g.C) + (slab + (long long)grow * g.ldc + col) * ELEM;
         if (col + PER <= lim) {
             if (RESIDUAL) red_add_v4_f32(reinterpret_cast<float *>(dst), v);
             else *reinterpret_cast<uint4 *>(dst) = v;
@@ -178,7 +181,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
                     park16(stage, lane, 4 * h, o);
                 }
                 __syncwarp();
-                flush_unit<2, false>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                flush_unit<2, false>(g, 0, stage, lane, grow0, M, t.ncol0 + c, lim);
                 __syncwarp();
             }
         } else if (g.vt != nullptr && t.ncol0 >= g.vt_col0) {
@@ -200,15 +203,15 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
                 uint32_t v[32];
                 tc::tmem_ld32(tbase + c, v);
                 tc::tmem_ld_wait();
-                if (g.mode != GEMM_RESIDUAL_F32) {
+                if (g.mode != GEMM_RESIDUAL_F32 && g.scale != 1.0f) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * g.scale);
                 }
                 park16(stage, lane, 0, v);
                 park16(stage, lane, 4, v + 16);
                 __syncwarp();
-                if (g.mode == GEMM_RESIDUAL_F32) flush_unit<4, true>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
-                else flush_unit<4, false>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                if (g.mode == GEMM_RESIDUAL_F32 && g.splits == 1) flush_unit<4, true>(g, 0, stage, lane, grow0, M, t.ncol0 + c, lim);
+                else flush_unit<4, false>(g, (long long)t.split * g.split_stride, stage, lane, grow0, M, t.ncol0 + c, lim);
                 __syncwarp();
             }
         } else {
@@ -223,7 +226,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
                     park16(stage, lane, 4 * h, o);
                 }
                 __syncwarp();
-                flush_unit<2, false>(g, stage, lane, grow0, M, t.ncol0 + c, lim);
+                flush_unit<2, false>(g, 0, stage, lane, grow0, M, t.ncol0 + c, lim);
                 __syncwarp();
             }
         }
@@ -239,7 +242,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
     const int MB = g.mb;
     const int m_groups = (M + MB * 2 * BM - 1) / (MB * 2 * BM);
-    const int num_tiles = m_groups * g.n_col_tiles;
+    const int num_tiles = m_groups * g.n_col_tiles * g.splits;
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
     if (pair >= num_tiles) return;
 
@@ -295,7 +298,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                                            : (t.map_idx == 0 ? &tmB0 : (t.map_idx == 1 ? &tmB1 : &tmB2));
             const int brow = swiglu ? t.n_local : t.n_local + (int)rank * HALF;
             const int arow = t.m0 + (int)rank * BM;
-            for (int kb = 0; kb < num_kb; ++kb, ++it) {
+            const int kb0 = t.split * g.kb_per_split, kb1 = min(num_kb, kb0 + g.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
                 const uint32_t s = it % (uint32_t)STAGES, ph = (it / (uint32_t)STAGES) & 1u;
                 if (!ready) ready = tc::mbar_wait(bar_empty + 8 * s, ph ^ 1u, &s_abort);
                 ok = __all_sync(0xffffffffu, ready);
@@ -331,7 +335,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 if (!ok) break;
                 tc::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + buf * buf_stride;
-                for (int kb = 0; kb < num_kb; ++kb, ++it) {
+                const int kb0 = tile_coord(g, tile, m_groups).split * g.kb_per_split, kb1 = min(num_kb, kb0 + g.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const uint32_t s = it % (uint32_t)STAGES, ph = (it / (uint32_t)STAGES) & 1u;
                     if (!ready) ready = tc::mbar_wait(bar_full + 8 * s, ph, &s_abort);
                     ok = __all_sync(0xffffffffu, ready);
@@ -341,7 +346,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     ready = tc::mbar_test(bar_full + 8 * ns, nph);
                     const uint32_t sa = smem_base + s * STAGE_BYTES;
                     const uint64_t da = tc::smem_desc_sw128(sa), db = tc::smem_desc_sw128(sa + MB * A_BYTES);
-                    const uint32_t acc = kb != 0 ? 1u : 0u;
+                    const uint32_t acc = kb != kb0 ? 1u : 0u;
                     tc::mma_bf16_2cta_elect(d_tmem, da, db, idesc, acc);
 #pragma unroll
                     for (int kk = 1; kk < BK / 16; ++kk) tc::mma_bf16_2cta_elect(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, 1u);
@@ -408,31 +413,37 @@ int stages_for(int mb, int bn)
     return s > kMaxStages ? kMaxStages : s;
 }
 
-// Tile shape (MB blocks of 256 rows, width bn): the candidate with the smallest modelled time
-//   waves x (k-blocks x max(MMA clocks, operand-stream clocks) + exposed epilogue clocks)
-// per pair of SMs.  Per k-block and CTA the tensor core needs MB*bn*2 clocks (8192 FLOP/clk/SM); the operand
-// stream is (MB*128 + bn/2) rows x 128 B at the ~40 B/clk an SM sustains from L2 when every SM streams (measured),
-// with a floor for the per-k-block handshakes.  The epilogue is hidden behind the next tile when two accumulators
-// fit tensor memory, except for the last tile of a pair.
-void pick_tile(int M, int K, int mode, int n_maps, int n_per_map, int pairs, int *mb_out, int *bn_out)
+// Modelled clocks of one candidate: waves x (k-blocks x clocks per k-block + exposed epilogue), per pair of SMs.
+// Per k-block and CTA the tensor core needs MB*bn*2 clocks (8192 FLOP/clk/SM); the operand stream is
+// (MB*128 + bn/2) rows x 128 B at the ~40 B/clk an SM sustains from L2 when every SM streams; below ~750 clocks the
+// k-block time stops shrinking with the tile (load latency over the bytes a CTA can keep in flight).  All measured.
+// The epilogue hides behind the next tile when two accumulators fit tensor memory, except for a pair's last tile.
+long long model_clocks(int M, int K, int mode, int n_maps, int n_per_map, int pairs, int mb, int bn, int splits)
+{
+    const long long num_kb = (K + BK - 1) / BK, kbps = (num_kb + splits - 1) / splits;
+    const int m_groups = (M + mb * 2 * BM - 1) / (mb * 2 * BM);
+    const long long tiles = (long long)m_groups * col_tiles(mode, n_maps, n_per_map, bn) * ((num_kb + kbps - 1) / kbps);
+    const long long waves = (tiles + pairs - 1) / pairs;
+    const long long mma = (long long)mb * bn * 2, load = (long long)(mb * BM + bn / 2) * 128 / 40;
+    long long kb_clk = mma > load ? mma : load;
+    if (kb_clk < 750) kb_clk = 750;
+    const long long epi = (long long)mb * bn * 16 + 3000;
+    const bool hidden = mb * ((bn + 31) & ~31) <= 256;
+    return waves * kbps * kb_clk + (hidden ? 1 : waves) * epi + (splits > 1 ? 1500LL * splits : 0);
+}
+
+// Tile shape (MB blocks of 256 rows, width bn) and number of K ranges with the smallest modelled time.  Wide, tall tiles
+// win when there are many tiles; narrower or shorter ones, or a split K, when a big tile would leave most pairs idle.
+void pick_tile(int M, int K, int mode, int n_maps, int n_per_map, int pairs, int max_splits, int *mb_out, int *bn_out, int *splits_out)
 {
     const int step = (mode == GEMM_SWIGLU) ? 32 : 16;
-    const long long num_kb = (K + BK - 1) / BK;
     long long best_cost = -1;
-    for (int mb = (M > 2 * BM ? 2 : 1); mb >= 1; --mb) {
-        const int m_groups = (M + mb * 2 * BM - 1) / (mb * 2 * BM);
-        for (int bn = 256; bn >= 32; bn -= step) {
-            const long long tiles = (long long)m_groups * col_tiles(mode, n_maps, n_per_map, bn);
-            const long long waves = (tiles + pairs - 1) / pairs;
-            const long long mma = (long long)mb * bn * 2, load = (long long)(mb * BM + bn / 2) * 128 / 40;
-            long long kb_clk = mma > load ? mma : load;
-            if (kb_clk < 450) kb_clk = 450;
-            const long long epi = (long long)mb * bn * 16 + 3000;
-            const bool hidden = mb * ((bn + 31) & ~31) <= 256;
-            const long long cost = waves * num_kb * kb_clk + (hidden ? 1 : waves) * epi;
-            if (best_cost < 0 || cost < best_cost) { best_cost = cost; *mb_out = mb; *bn_out = bn; }
-        }
-    }
+    for (int mb = (M > 2 * BM ? 2 : 1); mb >= 1; --mb)
+        for (int bn = 256; bn >= 32; bn -= step)
+            for (int sp = 1; sp <= max_splits; ++sp) {
+                const long long cost = model_clocks(M, K, mode, n_maps, n_per_map, pairs, mb, bn, sp);
+                if (best_cost < 0 || cost < best_cost) { best_cost = cost; *mb_out = mb; *bn_out = bn; *splits_out = sp; }
+            }
 }
 
 }  // namespace
@@ -449,7 +460,8 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     const int N = (mode == GEMM_SWIGLU) ? n_per_map : n_per_map * n_maps;
     SFS_REQUIRE(aligned_to(C, 16) && (ldc % 8) == 0, SFS_ERR_INVALID_ARG, "gemm: C must be 16-byte aligned, ldc a multiple of 8");
     int mb = 1, bn = 256;
-    pick_tile(M, K, mode, n_maps, n_per_map, num_sms() / 2, &mb, &bn);
+    int sp_unused = 1;
+    pick_tile(M, K, mode, n_maps, n_per_map, num_sms() / 2, 1, &mb, &bn, &sp_unused);
     if (tune) {                                              // measurement overrides; invalid values are ignored
         if (tune->mb == 1 || tune->mb == 2) mb = tune->mb;
         if (tune->bn >= 32 && tune->bn <= 256 && (tune->bn % ((mode == GEMM_SWIGLU) ? 32 : 16)) == 0) bn = tune->bn;
@@ -471,6 +483,40 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     g.stages = stages_for(mb, bn);
     if (tune && tune->stages >= 1 && tune->stages <= g.stages) g.stages = tune->stages;
     g.acc_bufs = (mb * ((bn + 31) & ~31) <= 256) ? 2 : 1;
+    g.splits = 1; g.kb_per_split = (K + BK - 1) / BK; g.split_stride = 0;
+    p->A = A; p->lda = lda; p->ldb = ldb;
+    for (int i = 0; i < 3; ++i) p->Bs[i] = Bs[i < n_maps ? i : 0];
+    return SFS_OK;
+}
+
+int32_t gemm_plan_enable_split(GemmPlan *p, float *ws, int32_t max_splits, const GemmTune *tune)
+{
+    GemmArgs &g = p->args;
+    if (g.mode != GEMM_RESIDUAL_F32 || ws == nullptr || max_splits < 2) return SFS_OK;
+    int mb = g.mb, bn = g.bn, sp = 1;
+    pick_tile(g.M, g.K, g.mode, p->n_maps, p->n_per_map, num_sms() / 2, max_splits, &mb, &bn, &sp);
+    if (tune) {
+        if (tune->mb == 1 || tune->mb == 2) mb = tune->mb;
+        if (tune->bn >= 32 && tune->bn <= 256 && (tune->bn % 16) == 0) bn = tune->bn;
+        if (tune->splits >= 1 && tune->splits <= max_splits) sp = tune->splits;
+    }
+    if (sp <= 1 && !tune) return SFS_OK;
+    // rebuild the plan at the new tile shape, then cut K
+    GemmPlan q;
+    GemmTune t2 = {mb, bn, tune ? tune->stages : 0, 0};
+    int32_t rc = gemm_plan_create(&q, p->A, p->lda, g.M, g.K, p->Bs, p->n_maps, p->n_per_map, p->ldb, g.mode, g.C, g.ldc, g.out_f32,
+                                  g.scale, g.vt, g.ldvt, g.vt_col0, &t2);
+    if (rc != SFS_OK) return rc;
+    *p = q;
+    GemmArgs &h = p->args;
+    const int num_kb = (h.K + BK - 1) / BK;
+    if (sp > num_kb) sp = num_kb;
+    if (sp > 1) {
+        h.kb_per_split = (num_kb + sp - 1) / sp;
+        h.splits = (num_kb + h.kb_per_split - 1) / h.kb_per_split;
+        h.split_stride = (long long)h.M * h.ldc;
+        h.C = ws;
+    }
     return SFS_OK;
 }
 
@@ -487,7 +533,7 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
     g.d_m = d_m; g.err = err; g.d_active = d_active;
     size_t smem = (size_t)g.stages * (g.mb * A_BYTES + (g.bn / 2) * BK * 2) + kBarBytes + kEpiStageBytes + 1024;
     if (smem < 120 * 1024) smem = 120 * 1024;
-    const long long tiles = (long long)((g.M + g.mb * 2 * BM - 1) / (g.mb * 2 * BM)) * g.n_col_tiles;
+    const long long tiles = (long long)((g.M + g.mb * 2 * BM - 1) / (g.mb * 2 * BM)) * g.n_col_tiles * g.splits;
     const int pairs = num_sms() / 2;
     dim3 grid((unsigned)(2 * (tiles < pairs ? tiles : pairs)), 1, 1);
     gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);

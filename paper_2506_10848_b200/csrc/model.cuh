@@ -25,6 +25,8 @@ struct sfs_session {
     int32_t *ticket = nullptr;               // [1]
     // forward workspace (model sessions only); T = max_batch*max_seq
     float *x = nullptr;                      // [T, d] fp32 residual stream
+    float *partial = nullptr;                // [kMaxSplits, T, d] split-K partial products of the residual projections
+    int pending_partials = 0;                // slabs the next RMSNorm must fold into x
     __nv_bfloat16 *h = nullptr;              // [T, d] normalised activations
     __nv_bfloat16 *qk = nullptr;             // [T, 2d] q | k
     __nv_bfloat16 *vt = nullptr;             // [d, T] V transposed
