@@ -83,3 +83,28 @@ def test_epilogue_microbenchmark_shape_full_size():
     # run-to-run determinism
     arg2, sq2, _ = gpu_stats(x.to(DEV), 126464, 126464, sfs.LOGITS_BF16)
     assert np.array_equal(sq, sq2) and np.array_equal(arg, arg2)
+
+
+def test_long_rows_special_values_padding_and_device_row_count():
+    """Rows long enough for the streaming kernel: padded leading dimension, -inf / tied / huge entries, a maximum in
+    the first and in the last column, and a device-side row count below the number of rows supplied."""
+    V, ld, R = 40008, 40960, 9
+    g = torch.Generator().manual_seed(7)
+    x = torch.randn((R, ld), generator=g) * 4
+    x[:, V:] = 1e30                                                      # padding beyond the vocabulary must be ignored
+    x[0, :V] = -float("inf"); x[0, 33333] = 1.5
+    x[1, :V] = 2.25                                                      # fully tied
+    x[2, 0] = 50.0
+    x[3, V - 1] = 50.0
+    x[4, 100] = 3e38; x[4, 101] = -3e38
+    x[5, :V] = -float("inf")
+    x[6, 20000] = x[6, :V].max(); x[6, 39999] = x[6, 20000]              # duplicated maximum: lowest id wins
+    xb = x.to(torch.bfloat16)
+    ref = RS.row_stats(np.ascontiguousarray(W.bf16_bits(xb)[:, :V]))
+    arg, sq, _ = gpu_stats(xb.to(DEV), V, ld, sfs.LOGITS_BF16)
+    assert np.array_equal(arg, ref["argmax"]) and np.array_equal(sq, ref["sq"])
+    n = torch.tensor([4], dtype=torch.int32, device=DEV)
+    arg, sq, _ = gpu_stats(xb.to(DEV), V, ld, sfs.LOGITS_BF16, n_rows_dev=n, max_rows=R)
+    assert np.array_equal(arg[:4], ref["argmax"][:4]) and np.array_equal(sq[:4], ref["sq"][:4])
+    assert np.all(arg[4:] == -7)
+    sfs.sfs_check_device_status()
