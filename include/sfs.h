@@ -184,6 +184,35 @@ int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_t logits_dt
                           int32_t *d_sel_count, int32_t *d_sel_pos, int32_t *d_sel_tok,
                           int32_t *d_next_rows, int32_t *d_next_n_rows, int32_t *d_trace, void *stream);
 
+/* ---- feature cache (optional) ------------------------------------------------------------------------- */
+
+/* The adaptive feature caching the paper's sampler integrates (Section 2.2; the (K_p, K_r) settings of Table 4).  The
+ * paper gives no mechanism, so the rule is this library's reading: per layer the cache holds every position's rotated
+ * key, value, and the residual increments of the attention and MLP branches.  Step t (from 0) recomputes the prompt
+ * positions when t mod k_prompt == 0 and all response positions when t mod k_response == 0; otherwise, per layer, the
+ * ceil(rho * gen_len) response positions whose fresh value vector is least similar (cosine) to the cached one (ties to
+ * the lower position; in a fast step only positions of the span [s_cycle, hi) are candidates).  Recomputed queries attend
+ * to all cached keys / values; every other position reuses its cached increments.  With k_prompt = k_response = 1 the
+ * result is the uncached forward pass. */
+typedef struct {
+    int32_t k_prompt;       /* 100  prompt refresh interval */
+    int32_t k_response;     /* 5    response refresh interval */
+    float   rho;            /* 0.25 fraction of the response recomputed on the other steps */
+} sfs_cache_params;
+
+/* Switches the cache on for the session (allocating per-layer caches for max_batch x max_seq tokens on the first call)
+ * and restarts the step counter; params == NULL switches it off.  sfs_generate* then runs cached steps. */
+int32_t sfs_cache_enable(sfs_session *session, const sfs_cache_params *params);
+/* Restarts the step counter: the next step recomputes everything. */
+int32_t sfs_cache_reset(sfs_session *session);
+/* One cached forward step (as sfs_forward, for B sequences of P prompt + (S - P) response tokens); advances the step
+ * counter.  d_state [B] (optional) tells slow from fast steps and gives the span; NULL means slow.  Optional dumps:
+ * d_sets int32 [n_layers, B, n_sel] receives the recomputed token indices of every layer (n_sel as returned in *n_sel,
+ * a HOST int), d_sims float [n_layers, B, S - P] the similarities (only written on adaptive steps). */
+int32_t sfs_forward_cached(sfs_session *session, const int32_t *d_tokens, int32_t B, int32_t S, int32_t P,
+                           const sfs_state *d_state, const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
+                           void *d_logits, int32_t logits_dtype, int32_t *d_sets, float *d_sims, int32_t *n_sel, void *stream);
+
 /* ---- the whole loop ------------------------------------------------------------------------------------ */
 
 /* Algorithm 1 for B independent sequences with a common prompt length P and response length gen_len:
@@ -221,7 +250,8 @@ int32_t sfs_generate_end(sfs_session *session, int32_t *d_out_tokens, sfs_state 
 #define SFS_K_GEMM_LM_HEAD 8
 #define SFS_K_ROW_STATS    9
 #define SFS_K_SELECT       10
-#define SFS_K_CLASSES      11
+#define SFS_K_CACHE        11   /* similarity, row choice, gathers and scatters of the feature cache */
+#define SFS_K_CLASSES      12
 
 /* Per-kernel timing of a session's forward / generate launches.  First synchronises the device and, when the
  * output pointers (HOST arrays of SFS_K_CLASSES entries) are not NULL, reports the milliseconds and launch

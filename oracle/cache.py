@@ -11,7 +11,7 @@ response's intermediate features across denoising steps and refreshes them at a 
   In layer l the set R_l of recomputed positions is
         prompt positions, if refresh_p;  plus
         all response positions, if refresh_r;  otherwise the adaptive set: with h = RMSNorm(x) and
-        v_i = h_i Wv^T for the candidate response positions C, the k = min(ceil(rho * L), |C|) candidates whose
+        v_i = h_i Wv^T for the candidate response positions C, the k = min(ceil(rho * L), |C|) candidates (rho as float32) whose
         cosine similarity  <v_i, V_l[i]> / (|v_i| |V_l[i]|)  to their cached value is smallest (ties: lower
         position first).  C is every response position in a slow step and the span [s_cycle, hi) in a fast
         step (out-of-span positions keep their cached features while the span is decoded).
@@ -53,6 +53,11 @@ def least_similar(sims: np.ndarray, candidates: Sequence[int], k: int) -> List[i
     return sorted(candidates[j] for j in order[:k])
 
 
+def adaptive_count(rho: float, L: int) -> int:
+    """ceil(rho * L) with rho taken as the float32 the interface carries (as the thresholds of the scheduler are)."""
+    return int(math.ceil(float(np.float32(rho)) * L))
+
+
 def cached_forward(cfg: F.ModelConfig, w: Dict, tokens: Sequence[int], P: int, cache: FeatureCache,
                    k_prompt: int, k_response: int, rho: float, span: Optional[Sequence[int]] = None,
                    rows: Optional[Sequence[int]] = None,
@@ -74,7 +79,7 @@ def cached_forward(cfg: F.ModelConfig, w: Dict, tokens: Sequence[int], P: int, c
     refresh_p = (cache.t % k_prompt) == 0
     refresh_r = (cache.t % k_response) == 0
     cand = list(range(L)) if span is None else list(range(span[0], span[1]))
-    k_adapt = min(int(math.ceil(rho * L)), len(cand))
+    k_adapt = min(adaptive_count(rho, L), len(cand))
     x = cast(w["tok_emb"])[tokens]                                   # [S, d]
     pos_all = np.arange(S)
     for l in range(cfg.n_layers):

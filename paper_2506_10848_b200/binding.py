@@ -42,6 +42,10 @@ class Params(Structure):
         return p
 
 
+class CacheParams(Structure):
+    _fields_ = [("k_prompt", c_int32), ("k_response", c_int32), ("rho", c_float)]
+
+
 STATE_INTS = 32
 STATE_FIELDS = ["phase", "s_cycle", "hi", "step_count", "hist_len"] + [f"hist{i}" for i in range(MAX_W_HIST)] + \
                ["k_remaining", "n_masked", "steps_done", "n_slow", "n_fast", "n_cycles", "n_fallback", "done", "status"]
@@ -183,6 +187,28 @@ def sfs_forward(session, tokens, B, S, rows, n_rows_dev, max_rows, logits, logit
                              _ptr(logits), c_int32(logits_dtype), _stream(stream)))
 
 
+def sfs_cache_enable(session, k_prompt=100, k_response=5, rho=0.25, off=False):
+    if off:
+        _check(lib().sfs_cache_enable(session, None))
+        return
+    p = CacheParams(int(k_prompt), int(k_response), float(rho))
+    _check(lib().sfs_cache_enable(session, byref(p)))
+
+
+def sfs_cache_reset(session):
+    _check(lib().sfs_cache_reset(session))
+
+
+def sfs_forward_cached(session, tokens, B, S, P, state, rows, n_rows_dev, max_rows, logits, logits_dtype, sets=None, sims=None,
+                       stream=None):
+    """Returns n_sel, the number of recomputed rows per sequence and layer in this step."""
+    n = c_int32(0)
+    _check(lib().sfs_forward_cached(session, _ptr(tokens), c_int32(B), c_int32(S), c_int32(P), _ptr(state), _ptr(rows), _ptr(n_rows_dev),
+                                    c_int32(max_rows), _ptr(logits), c_int32(logits_dtype), _ptr(sets), _ptr(sims), byref(n),
+                                    _stream(stream)))
+    return n.value
+
+
 def sfs_generate(session, prompt, B, P, gen_len, params, out_tokens, state_out=None, trace=None, max_trace_steps=0, stream=None):
     _check(lib().sfs_generate(session, _ptr(prompt), c_int32(B), c_int32(P), c_int32(gen_len), byref(params), _ptr(out_tokens),
                               _ptr(state_out), _ptr(trace), c_int32(max_trace_steps), _stream(stream)))
@@ -205,7 +231,7 @@ def sfs_generate_end(session, out_tokens=None, state_out=None, stream=None):
 
 
 K_CLASSES = ["embed", "rmsnorm", "gemm_qkv", "rope", "attention", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_lm_head",
-             "row_stats", "select"]
+             "row_stats", "select", "cache"]
 
 
 def sfs_profile(session, enable, read=True):

@@ -5,6 +5,8 @@
 #include "gemm.cuh"
 #include "attention.cuh"
 #include "elementwise.cuh"
+#include "cache.cuh"
+#include <math.h>
 
 #include <new>
 #include <string.h>
@@ -135,7 +137,7 @@ static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int3
         const LayerPlans &lp = s->layer_plans[l];
         if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, pending, pstride, m->attn_norm[l], s->h, nullptr, nullptr, T, d, c.rms_eps, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(lp.qkv, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-        if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, st); })) != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, nullptr, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch(s->attn_plan, d_active, err, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(lp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
         pending = lp.o.args.splits > 1 ? lp.o.args.splits : 0;
@@ -144,7 +146,165 @@ static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int3
         if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(lp.down, nullptr, d_active, err, st); })) != SFS_OK) return rc;
         pending = lp.down.args.splits > 1 ? lp.down.args.splits : 0;
     }
-    s->pending_partials = pending;                           // for the final RMSNorm of the caller
+    s->pending_ptr = s->partial; s->pending_n = pending; s->pending_stride = pstride;      // for the final RMSNorm of the caller
+    return SFS_OK;
+}
+
+// ---- cached steps --------------------------------------------------------------------------------------
+// per-layer plans of the cached mode that do not depend on the number of recomputed rows
+static int32_t cache_plan(sfs_session *s, int32_t B, int32_t S)
+{
+    const sfs_model *m = s->model;
+    const sfs_config &c = m->cfg;
+    const int T = B * S, d = c.d_model, ff = c.d_ff;
+    if ((int)s->cache_plans.size() == c.n_layers && s->cache_B == B && s->cache_S == S) return SFS_OK;
+    s->cache_plans.assign(c.n_layers, CacheLayerPlans());
+    s->gather_plans.clear();
+    int32_t rc;
+    for (int l = 0; l < c.n_layers; ++l) {
+        CacheLayerPlans &cp = s->cache_plans[l];
+        const void *wv[1] = {m->wv[l]};
+        // fresh values of every row, written transposed (every output column goes through the transposed store)
+        rc = gemm_plan_create(&cp.vproj, s->h, d, T, d, wv, 1, d, d, GEMM_STORE, s->attn, d, 0, 1.0f, s->vnew_t, T, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+        const void *wo[1] = {m->wo[l]};
+        rc = gemm_plan_create(&cp.o_store, s->attn, d, T, d, wo, 1, d, d, GEMM_STORE, s->Ac[l], d, 1, 1.0f, nullptr, 0, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+        const void *wd[1] = {m->w_down[l]};
+        rc = gemm_plan_create(&cp.down_store, s->hid, ff, T, ff, wd, 1, d, ff, GEMM_STORE, s->Fc[l], d, 1, 1.0f, nullptr, 0, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+        rc = attn_plan_create_split(&cp.attn, s->qk, 2 * d, s->Kc[l], d, d, 0, s->Vtc[l], T, s->attn, d, B, S, c.n_heads, c.head_dim);
+        if (rc != SFS_OK) return rc;
+    }
+    return SFS_OK;
+}
+
+// projections over the compact buffers of NR recomputed rows
+static int32_t gather_plan(sfs_session *s, int32_t NR, int32_t T, std::vector<GatherLayerPlans> **out)
+{
+    auto it = s->gather_plans.find(NR);
+    if (it != s->gather_plans.end()) { *out = &it->second; return SFS_OK; }
+    const sfs_model *m = s->model;
+    const sfs_config &c = m->cfg;
+    const int d = c.d_model, ff = c.d_ff;
+    std::vector<GatherLayerPlans> v(c.n_layers);
+    int32_t rc;
+    for (int l = 0; l < c.n_layers; ++l) {
+        GatherLayerPlans &gp = v[l];
+        const void *qkv[3] = {m->wq[l], m->wk[l], m->wv[l]};
+        rc = gemm_plan_create(&gp.qkv, s->hg, d, NR, d, qkv, 3, d, d, GEMM_STORE, s->qk, 2 * d, 0, 1.0f, s->vt, T, 2 * d, nullptr);
+        if (rc != SFS_OK) return rc;
+        const void *wo[1] = {m->wo[l]};
+        rc = gemm_plan_create(&gp.o, s->attn, d, NR, d, wo, 1, d, d, GEMM_STORE, s->partial, d, 1, 1.0f, nullptr, 0, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+        const void *gu[2] = {m->w_gate[l], m->w_up[l]};
+        rc = gemm_plan_create(&gp.gate_up, s->hg, d, NR, d, gu, 2, ff, d, GEMM_SWIGLU, s->hid, ff, 0, 1.0f, nullptr, 0, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+        const void *wd[1] = {m->w_down[l]};
+        rc = gemm_plan_create(&gp.down, s->hid, ff, NR, ff, wd, 1, d, ff, GEMM_STORE, s->partial, d, 1, 1.0f, nullptr, 0, 0, nullptr);
+        if (rc != SFS_OK) return rc;
+    }
+    auto ins = s->gather_plans.emplace(NR, std::move(v));
+    *out = &ins.first->second;
+    return SFS_OK;
+}
+
+// One cached step of the transformer body (the rule is stated with sfs_cache_params in sfs.h): tokens -> x [T, d],
+// leaving the last layer's MLP increment pending for the caller's final RMSNorm.
+static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t S, int32_t P, const sfs_state *d_state,
+                               const int32_t *d_active, int32_t *d_sets, float *d_sims, int32_t *n_sel_out, cudaStream_t st)
+{
+    const sfs_model *m = s->model;
+    const sfs_config &c = m->cfg;
+    const int T = B * S, L = S - P, d = c.d_model;
+    SFS_REQUIRE(s->cache_on, SFS_ERR_INVALID_ARG, "cached step: call sfs_cache_enable first");
+    SFS_REQUIRE(P >= 0 && L >= 1, SFS_ERR_INVALID_ARG, "cached step: P=%d S=%d", P, S);
+    if (s->cache_t != 0)
+        SFS_REQUIRE(s->cache_B == B && s->cache_S == S && s->cache_P == P, SFS_ERR_INVALID_ARG,
+                    "cached step: the cached features belong to B=%d S=%d P=%d; call sfs_cache_reset before changing the shape",
+                    s->cache_B, s->cache_S, s->cache_P);
+    int32_t *err = device_status_word();
+    SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
+    int32_t rc;
+    if ((rc = session_plan(s, B, S)) != SFS_OK) return rc;
+    if ((rc = cache_plan(s, B, S)) != SFS_OK) return rc;
+    s->cache_B = B; s->cache_S = S; s->cache_P = P;
+    const sfs_cache_params &cp = s->cache_params;
+    const bool rp = (s->cache_t % cp.k_prompt) == 0, rr = (s->cache_t % cp.k_response) == 0;
+    int n_adapt = (int)ceil((double)cp.rho * (double)L);
+    n_adapt = n_adapt < 0 ? 0 : (n_adapt > L ? L : n_adapt);
+    const int n_sel = (rp ? P : 0) + (rr ? L : n_adapt);
+    if (n_sel_out) *n_sel_out = (rp && rr) ? S : n_sel;
+    const int NR = B * n_sel;
+
+    if ((rc = timed_launch(s, SFS_K_EMBED, st, [&] { return launch_embed(d_tokens, m->tok_emb, s->x, T, d, c.vocab, st); })) != SFS_OK) return rc;
+    const float *pend = nullptr;
+    auto norm_all = [&](const void *gain) {
+        return timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, pend, pend ? 1 : 0, 0, gain, s->h, nullptr, nullptr, T, d, c.rms_eps, st); });
+    };
+    if (rp && rr) {
+        // everything is recomputed: the uncached layer pipeline, with the increments stored instead of added and K / V copied out
+        for (int l = 0; l < c.n_layers; ++l) {
+            const LayerPlans &lp = s->layer_plans[l];
+            const CacheLayerPlans &cl = s->cache_plans[l];
+            if ((rc = norm_all(m->attn_norm[l])) != SFS_OK) return rc;
+            if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(lp.qkv, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+            if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, T, S, c.n_heads, c.head_dim, s->rope_table, nullptr, st); })) != SFS_OK) return rc;
+            SFS_CUDA(cudaMemcpy2DAsync(s->Kc[l], (size_t)d * 2, s->qk + d, (size_t)2 * d * 2, (size_t)d * 2, (size_t)T, cudaMemcpyDeviceToDevice, st));
+            SFS_CUDA(cudaMemcpyAsync(s->Vtc[l], s->vt, (size_t)d * T * 2, cudaMemcpyDeviceToDevice, st));
+            if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch(s->attn_plan, d_active, err, st); })) != SFS_OK) return rc;
+            if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(cl.o_store, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+            pend = s->Ac[l];
+            if ((rc = norm_all(m->mlp_norm[l])) != SFS_OK) return rc;
+            if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(lp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+            if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(cl.down_store, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+            pend = s->Fc[l];
+            if (d_sets) {   // the dump lists every token
+                CacheSelectArgs a{}; a.B = B; a.S = S; a.P = P; a.L = L; a.T = T; a.refresh_p = 1; a.refresh_r = 1; a.n_sel = S;
+                a.sel_rows = d_sets + (size_t)l * B * S;
+                if ((rc = launch_cache_select(a, st)) != SFS_OK) return rc;
+            }
+        }
+    } else {
+        std::vector<GatherLayerPlans> *gps = nullptr;
+        if (NR > 0 && (rc = gather_plan(s, NR, T, &gps)) != SFS_OK) return rc;
+        for (int l = 0; l < c.n_layers; ++l) {
+            const CacheLayerPlans &cl = s->cache_plans[l];
+            if ((rc = norm_all(m->attn_norm[l])) != SFS_OK) return rc;
+            if (NR > 0) {
+                const GatherLayerPlans &gp = (*gps)[l];
+                if (!rr && n_adapt > 0) {
+                    if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(cl.vproj, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+                    if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_sim_partial(s->vnew_t, s->Vtc[l], T, d, T, s->sim_partial, st); })) != SFS_OK) return rc;
+                }
+                CacheSelectArgs a{};
+                a.partial = s->sim_partial; a.state = d_state; a.B = B; a.S = S; a.P = P; a.L = L; a.T = T;
+                a.refresh_p = rp; a.refresh_r = rr; a.n_adapt = rr ? 0 : n_adapt; a.n_sel = n_sel; a.sel_rows = s->sel_rows;
+                a.sims_dump = (d_sims && !rr) ? d_sims + (size_t)l * B * L : nullptr;
+                a.sets_dump = d_sets ? d_sets + (size_t)l * NR : nullptr;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_cache_select(a, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_gather_rows_bf16(s->h, s->sel_rows, NR, d, s->hg, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(gp.qkv, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, NR, S, c.n_heads, c.head_dim, s->rope_table, s->sel_rows, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_kv(s->qk, 2 * d, d, s->vt, T, s->sel_rows, NR, d, s->Kc[l], s->Vtc[l], T, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch_queries(cl.attn, n_sel, d_active, err, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(gp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, s->sel_rows, NR, d, s->Ac[l], st); })) != SFS_OK) return rc;
+            }
+            pend = s->Ac[l];
+            if ((rc = norm_all(m->mlp_norm[l])) != SFS_OK) return rc;
+            if (NR > 0) {
+                const GatherLayerPlans &gp = (*gps)[l];
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_gather_rows_bf16(s->h, s->sel_rows, NR, d, s->hg, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(gp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(gp.down, nullptr, d_active, err, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, s->sel_rows, NR, d, s->Fc[l], st); })) != SFS_OK) return rc;
+            }
+            pend = s->Fc[l];
+        }
+    }
+    s->pending_ptr = pend; s->pending_n = pend ? 1 : 0; s->pending_stride = 0;
+    s->cache_t++;
     return SFS_OK;
 }
 
@@ -330,7 +490,7 @@ int32_t sfs_forward(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t 
     int32_t rc = session_plan(s, B, S);
     if (rc != SFS_OK) return rc;
     if ((rc = run_body(s, d_tokens, B, S, nullptr, st)) != SFS_OK) return rc;
-    if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, s->pending_partials, (long long)B * S * c.d_model, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
+    if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->pending_ptr, s->pending_n, s->pending_stride, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
     GemmPlan lm;
     const void *lmw[1] = {s->model->lm_head};
     rc = gemm_plan_create(&lm, s->hfin, c.d_model, max_rows, c.d_model, lmw, 1, c.vocab, c.d_model, GEMM_STORE, d_logits, c.vocab,
@@ -394,6 +554,68 @@ int32_t sfs_select(sfs_session *s, const void *d_logits, int32_t logits_dtype, i
     return launch_select(a, st);
 }
 
+// ---- feature cache ----------------------------------------------------------------------------------------
+int32_t sfs_cache_enable(sfs_session *s, const sfs_cache_params *p)
+{
+    SFS_REQUIRE(s && s->model, SFS_ERR_INVALID_ARG, "cache_enable: needs a session created from a model");
+    if (p == nullptr) { s->cache_on = false; return SFS_OK; }
+    SFS_REQUIRE(p->k_prompt >= 1 && p->k_response >= 1 && p->rho >= 0.f && p->rho <= 1.f, SFS_ERR_INVALID_ARG,
+                "cache_enable: k_prompt %d, k_response %d must be >= 1 and rho %g within [0, 1]", p->k_prompt, p->k_response, (double)p->rho);
+    const sfs_config &c = s->model->cfg;
+    const size_t T = (size_t)s->max_batch * s->max_seq, d = c.d_model;
+    if (s->Kc.empty()) {
+        int32_t rc;
+        s->Kc.resize(c.n_layers); s->Vtc.resize(c.n_layers); s->Ac.resize(c.n_layers); s->Fc.resize(c.n_layers);
+        for (int l = 0; l < c.n_layers; ++l) {
+            if ((rc = dev_alloc(s, &s->Kc[l], T * d, true)) != SFS_OK) return rc;
+            if ((rc = dev_alloc(s, &s->Vtc[l], T * d, true)) != SFS_OK) return rc;
+            if ((rc = dev_alloc(s, &s->Ac[l], T * d, true)) != SFS_OK) return rc;
+            if ((rc = dev_alloc(s, &s->Fc[l], T * d, true)) != SFS_OK) return rc;
+        }
+        if ((rc = dev_alloc(s, &s->hg, T * d, true)) != SFS_OK) return rc;
+        if ((rc = dev_alloc(s, &s->vnew_t, T * d, true)) != SFS_OK) return rc;
+        if ((rc = dev_alloc(s, &s->sim_partial, (size_t)kSimSlices * T * 3, true)) != SFS_OK) return rc;
+        if ((rc = dev_alloc(s, &s->sel_rows, T, true)) != SFS_OK) return rc;
+        SFS_CUDA(cudaDeviceSynchronize());
+    }
+    s->cache_params = *p;
+    s->cache_on = true;
+    s->cache_t = 0;
+    return SFS_OK;
+}
+
+int32_t sfs_cache_reset(sfs_session *s)
+{
+    SFS_REQUIRE(s != nullptr, SFS_ERR_INVALID_ARG, "cache_reset: session is NULL");
+    s->cache_t = 0;
+    return SFS_OK;
+}
+
+int32_t sfs_forward_cached(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t S, int32_t P,
+                           const sfs_state *d_state, const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
+                           void *d_logits, int32_t logits_dtype, int32_t *d_sets, float *d_sims, int32_t *n_sel, void *stream)
+{
+    SFS_REQUIRE(s && s->model, SFS_ERR_INVALID_ARG, "forward_cached: needs a session created from a model");
+    SFS_REQUIRE(d_tokens && d_logits, SFS_ERR_INVALID_ARG, "forward_cached: NULL device pointer");
+    SFS_REQUIRE(B >= 1 && B <= s->max_batch && S >= 8 && S <= s->max_seq && P >= 0 && P < S, SFS_ERR_INVALID_ARG,
+                "forward_cached: B=%d S=%d P=%d outside the session's limits (%d, %d)", B, S, P, s->max_batch, s->max_seq);
+    SFS_REQUIRE(max_rows >= 1 && max_rows <= B * S, SFS_ERR_INVALID_ARG, "forward_cached: max_rows %d outside [1, B*S]", max_rows);
+    SFS_REQUIRE(logits_dtype == SFS_LOGITS_BF16 || logits_dtype == SFS_LOGITS_F32, SFS_ERR_INVALID_ARG, "logits_dtype %d", logits_dtype);
+    SFS_REQUIRE(d_rows != nullptr || (max_rows == B * S && d_n_rows == nullptr), SFS_ERR_INVALID_ARG,
+                "forward_cached: without a row list all B*S rows are produced");
+    cudaStream_t st = (cudaStream_t)stream;
+    const sfs_config &c = s->model->cfg;
+    int32_t rc = run_body_cached(s, d_tokens, B, S, P, d_state, nullptr, d_sets, d_sims, n_sel, st);
+    if (rc != SFS_OK) return rc;
+    if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->pending_ptr, s->pending_n, s->pending_stride, s->model->final_norm, s->hfin, d_rows, d_n_rows, max_rows, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
+    GemmPlan lm;
+    const void *lmw[1] = {s->model->lm_head};
+    rc = gemm_plan_create(&lm, s->hfin, c.d_model, max_rows, c.d_model, lmw, 1, c.vocab, c.d_model, GEMM_STORE, d_logits, c.vocab,
+                          logits_dtype == SFS_LOGITS_F32 ? 1 : 0, c.logit_scale, nullptr, 0, 0, nullptr);
+    if (rc != SFS_OK) return rc;
+    return timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(lm, d_n_rows, nullptr, device_status_word(), st); });
+}
+
 // ---- the whole loop -------------------------------------------------------------------------------------
 int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, int32_t P, int32_t gen_len,
                            const sfs_params *params, void *stream)
@@ -421,6 +643,7 @@ int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, i
     s->gen_B = B; s->gen_P = P; s->gen_L = gen_len; s->gen_cur = 0; s->gen_steps = 0;
     s->gen_max_steps = params->max_steps > 0 ? params->max_steps : gen_len;
     s->gen_params = *params;
+    s->cache_t = 0;                                          // a new generation starts with a full refresh
     s->generating = true;
     *s->host_active = B;
     return SFS_OK;
@@ -442,8 +665,10 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         const int cur = s->gen_cur, nxt = cur ^ 1;
         const int32_t *d_active = s->ctrl + 2;
         const int32_t *rows = s->rows[cur], *n_rows = s->ctrl + cur;
-        if ((rc = run_body(s, s->tokens, B, S, d_active, st)) != SFS_OK) return rc;
-        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->partial, s->pending_partials, (long long)B * S * c.d_model, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
+        if (s->cache_on) rc = run_body_cached(s, s->tokens, B, S, P, s->state, d_active, nullptr, nullptr, nullptr, st);
+        else rc = run_body(s, s->tokens, B, S, d_active, st);
+        if (rc != SFS_OK) return rc;
+        if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->pending_ptr, s->pending_n, s->pending_stride, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_GEMM_LM_HEAD, st, [&] { return gemm_launch(s->lm_plan, n_rows, d_active, err, st); })) != SFS_OK) return rc;
         if (d_logits_dump) {
             SFS_CUDA(cudaMemcpyAsync(d_logits_dump, s->logits, (size_t)B * L * c.vocab * 2, cudaMemcpyDeviceToDevice, st));

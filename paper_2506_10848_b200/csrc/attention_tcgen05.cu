@@ -21,7 +21,7 @@ constexpr int KV_STAGES = 2;
 
 template <int DH>
 __global__ void __launch_bounds__(kAttnThreads, 1)
-attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant__ CUtensorMap tmVt, AttnArgs a)
+attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmVt, AttnArgs a)
 {
     constexpr int KB = DH / 64;                          // 64-element K-blocks along the head dimension
     constexpr int Q_BYTES = QT * DH * 2;
@@ -41,8 +41,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q0 = blockIdx.x * QT, h = blockIdx.y, b = blockIdx.z;
-    const int S = a.S, d = a.d_model;
-    const int tok0 = b * S;                                // first token of this sequence
+    const int S = a.S;
+    const int tok0 = b * S;                                // first key / value token of this sequence
+    const int qrow0 = b * a.kq + q0;                       // first query row of this CTA (queries may be a compact subset)
     const int nkv = (S + KT - 1) / KT;
 
     const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * KV_STAGES;
@@ -67,7 +68,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant
             tc::mbar_expect_tx(bar_q, Q_BYTES);
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
-                tc::tma_load_2d(tc::smem_u32(sQ) + kb * (QT * 128), &tmQK, h * DH + kb * 64, tok0 + q0, bar_q);
+                tc::tma_load_2d(tc::smem_u32(sQ) + kb * (QT * 128), &tmQ, h * DH + kb * 64, qrow0, bar_q);
             int issued = 0;
             for (int j = 0; j < nkv; ++j) {
                 const int s = j % KV_STAGES;
@@ -77,7 +78,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant
                 tc::mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
-                    tc::tma_load_2d(sk + kb * (KT * 128), &tmQK, d + h * DH + kb * 64, tok0 + j * KT, bar_full + 8 * s);
+                    tc::tma_load_2d(sk + kb * (KT * 128), &tmK, a.k_col0 + h * DH + kb * 64, tok0 + j * KT, bar_full + 8 * s);
 #pragma unroll
                 for (int kb = 0; kb < KT / 64; ++kb)
                     tc::tma_load_2d(sv + kb * (DH * 128), &tmVt, tok0 + j * KT + kb * 64, h * DH, bar_full + 8 * s);
@@ -209,9 +210,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant
             }
             tc::tc_fence_before();
         }
-        if (ok && !s_abort && q0 + row < S) {
+        if (ok && !s_abort && q0 + row < a.kq) {
             const float inv = 1.0f / l;
-            __nv_bfloat16 *dst = a.out + (long long)(tok0 + q0 + row) * a.ld_out + h * DH;
+            __nv_bfloat16 *dst = a.out + (long long)(qrow0 + row) * a.ld_out + h * DH;
 #pragma unroll
             for (int i = 0; i < DH / 8; ++i) {
                 uint32_t o[4];
@@ -232,7 +233,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQK, const __grid_constant
 }
 
 template <int DH>
-int32_t launch_dh(const AttnPlan &p, const int32_t *d_active, int32_t *err, cudaStream_t stream)
+int32_t launch_dh(const AttnPlan &p, int kq, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
     constexpr size_t smem = (size_t)QT * DH * 2 + KV_STAGES * (size_t)(KT * DH * 2 + DH * KT * 2) + QT * KT * 2
                           + (2 * KV_STAGES + 4) * 8 + 16 + 1024;
@@ -243,38 +244,53 @@ int32_t launch_dh(const AttnPlan &p, const int32_t *d_active, int32_t *err, cuda
     }
     AttnArgs a = p.args;
     a.err = err; a.d_active = d_active;
-    dim3 grid((unsigned)((a.S + QT - 1) / QT), (unsigned)a.n_heads, (unsigned)a.B);
-    attention_kernel<DH><<<grid, kAttnThreads, smem, stream>>>(p.tmQK, p.tmVt, a);
+    if (kq > 0) a.kq = kq;
+    dim3 grid((unsigned)((a.kq + QT - 1) / QT), (unsigned)a.n_heads, (unsigned)a.B);
+    attention_kernel<DH><<<grid, kAttnThreads, smem, stream>>>(p.tmQ, p.tmK, p.tmVt, a);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }
 
 }  // namespace
 
-int32_t attn_plan_create(AttnPlan *p, const void *qkv, int64_t ld_qkv, const void *vt, int64_t ld_vt,
-                         void *out, int64_t ld_out, int32_t B, int32_t S, int32_t n_heads, int32_t head_dim)
+int32_t attn_plan_create_split(AttnPlan *p, const void *q, int64_t ld_q, const void *k, int64_t ld_k, int32_t k_cols, int32_t k_col0,
+                               const void *vt, int64_t ld_vt, void *out, int64_t ld_out, int32_t B, int32_t S, int32_t n_heads, int32_t head_dim)
 {
     SFS_REQUIRE(head_dim == 64 || head_dim == 128, SFS_ERR_UNSUPPORTED, "attention: head_dim %d (64 or 128 supported)", head_dim);
     SFS_REQUIRE((S % 8) == 0, SFS_ERR_UNSUPPORTED, "attention: sequence length %d must be a multiple of 8", S);
     SFS_REQUIRE(aligned_to(out, 16) && (ld_out % 8) == 0, SFS_ERR_INVALID_ARG, "attention: output must be 16-byte aligned");
     memset(p, 0, sizeof(*p));
     const int d = n_heads * head_dim;
-    int32_t rc = make_tmap_bf16(&p->tmQK, qkv, (uint64_t)B * S, (uint64_t)2 * d, (uint64_t)ld_qkv, 128);
+    int32_t rc = make_tmap_bf16(&p->tmQ, q, (uint64_t)B * S, (uint64_t)d, (uint64_t)ld_q, 128);
+    if (rc != SFS_OK) return rc;
+    rc = make_tmap_bf16(&p->tmK, k, (uint64_t)B * S, (uint64_t)k_cols, (uint64_t)ld_k, 128);
     if (rc != SFS_OK) return rc;
     rc = make_tmap_bf16(&p->tmVt, vt, (uint64_t)d, (uint64_t)B * S, (uint64_t)ld_vt, (uint32_t)head_dim);
     if (rc != SFS_OK) return rc;
     AttnArgs &a = p->args;
-    a.B = B; a.S = S; a.n_heads = n_heads; a.d_model = d;
+    a.B = B; a.S = S; a.n_heads = n_heads; a.d_model = d; a.kq = S; a.k_col0 = k_col0;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)head_dim);
     a.out = reinterpret_cast<__nv_bfloat16 *>(out); a.ld_out = ld_out;
     p->head_dim = head_dim;
     return SFS_OK;
 }
 
+int32_t attn_plan_create(AttnPlan *p, const void *qkv, int64_t ld_qkv, const void *vt, int64_t ld_vt,
+                         void *out, int64_t ld_out, int32_t B, int32_t S, int32_t n_heads, int32_t head_dim)
+{
+    const int d = n_heads * head_dim;
+    return attn_plan_create_split(p, qkv, ld_qkv, qkv, ld_qkv, 2 * d, d, vt, ld_vt, out, ld_out, B, S, n_heads, head_dim);
+}
+
 int32_t attn_launch(const AttnPlan &p, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
-    if (p.head_dim == 128) return launch_dh<128>(p, d_active, err, stream);
-    return launch_dh<64>(p, d_active, err, stream);
+    return attn_launch_queries(p, 0, d_active, err, stream);
+}
+
+int32_t attn_launch_queries(const AttnPlan &p, int32_t kq, const int32_t *d_active, int32_t *err, cudaStream_t stream)
+{
+    if (p.head_dim == 128) return launch_dh<128>(p, kq, d_active, err, stream);
+    return launch_dh<64>(p, kq, d_active, err, stream);
 }
 
 }  // namespace sfs

@@ -1,0 +1,185 @@
+// Feature cache of the mask predictor (the adaptive caching the paper's sampler integrates, Section 2.2 and the
+// (K_p, K_r) settings of Table 4): value-similarity sums, the least-similar row choice, and the gathers / scatters
+// that move the recomputed rows between the compact buffers the GEMMs work on and the per-layer caches.
+#include "sfs_common.cuh"
+#include "cache.cuh"
+
+namespace sfs {
+namespace {
+
+// grid (ceil(T / 64), kSimSlices), 256 threads: lane = two neighbouring tokens, warp = every 8th feature of the slice
+__global__ void __launch_bounds__(256)
+sim_partial_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b, long long ld, int d, int T,
+                   float *__restrict__ partial)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int t0 = blockIdx.x * 64 + 2 * lane;
+    const int per = (d + kSimSlices - 1) / kSimSlices;
+    const int f0 = blockIdx.y * per, f1 = min(d, f0 + per);
+    float acc[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    if (t0 < T) {
+        for (int f = f0 + warp; f < f1; f += 8) {
+            const uint32_t wa = *reinterpret_cast<const uint32_t *>(a + (long long)f * ld + t0);
+            const uint32_t wb = *reinterpret_cast<const uint32_t *>(b + (long long)f * ld + t0);
+            const float a0 = bf16_bits_to_f32(wa & 0xFFFFu), a1 = bf16_bits_to_f32(wa >> 16);
+            const float b0 = bf16_bits_to_f32(wb & 0xFFFFu), b1 = bf16_bits_to_f32(wb >> 16);
+            acc[0] = fmaf(a0, b0, acc[0]); acc[1] = fmaf(a0, a0, acc[1]); acc[2] = fmaf(b0, b0, acc[2]);
+            acc[3] = fmaf(a1, b1, acc[3]); acc[4] = fmaf(a1, a1, acc[4]); acc[5] = fmaf(b1, b1, acc[5]);
+        }
+    }
+    __shared__ float s[8][32][6];
+#pragma unroll
+    for (int i = 0; i < 6; ++i) s[warp][lane][i] = acc[i];
+    __syncthreads();
+    if (warp == 0 && t0 < T) {
+        float r[6];
+#pragma unroll
+        for (int i = 0; i < 6; ++i) { r[i] = s[0][lane][i]; for (int w = 1; w < 8; ++w) r[i] += s[w][lane][i]; }   // fixed order
+        float *o = partial + ((long long)blockIdx.y * T + t0) * 3;
+        o[0] = r[0]; o[1] = r[1]; o[2] = r[2];
+        if (t0 + 1 < T) { o[3] = r[3]; o[4] = r[4]; o[5] = r[5]; }
+    }
+}
+
+__device__ __forceinline__ uint32_t float_order_key(float f) {       // monotone map float -> uint32
+    const uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+// one CTA per sequence; dynamic shared memory: u64 keys[L], u8 chosen[L]
+__global__ void __launch_bounds__(256) cache_select_kernel(CacheSelectArgs a)
+{
+    extern __shared__ unsigned long long s_key[];
+    const int b = blockIdx.x, tid = threadIdx.x, L = a.L, P = a.P, S = a.S;
+    int32_t *out = a.sel_rows + (long long)b * a.n_sel;
+    int base = 0;
+    if (a.refresh_p) {
+        for (int i = tid; i < P; i += blockDim.x) out[i] = b * S + i;
+        base = P;
+    }
+    if (a.refresh_r) {
+        for (int i = tid; i < L; i += blockDim.x) out[base + i] = b * S + P + i;
+    } else if (a.n_adapt > 0) {
+        int lo = 0, hi = L;
+        if (a.state != nullptr && a.state[b].phase == SFS_PHASE_FAST && !a.state[b].done) { lo = a.state[b].s_cycle; hi = a.state[b].hi; }
+        lo = max(0, min(lo, L)); hi = max(lo, min(hi, L));
+        for (int i = tid; i < L; i += blockDim.x) {
+            float dot = 0.f, na = 0.f, nb = 0.f;
+            const long long t = (long long)b * S + P + i;
+            for (int sl = 0; sl < kSimSlices; ++sl) {                // fixed order
+                const float *p = a.partial + ((long long)sl * a.T + t) * 3;
+                dot += p[0]; na += p[1]; nb += p[2];
+            }
+            const float den = __fmul_rn(__fsqrt_rn(na), __fsqrt_rn(nb));
+            const float sim = den > 0.f ? __fdiv_rn(dot, den) : 0.f;
+            if (a.sims_dump) a.sims_dump[(long long)b * L + i] = sim;
+            s_key[i] = (i >= lo && i < hi) ? (((unsigned long long)float_order_key(sim) << 32) | (unsigned)i) : ~0ull;
+        }
+        __syncthreads();
+        const int n_cand = hi - lo;
+        const int k = min(a.n_adapt, n_cand);
+        __shared__ int s_last;
+        if (tid == 0) s_last = -1;
+        __syncthreads();
+        // rank by counting: candidate i is chosen when fewer than k candidate keys are smaller
+        uint8_t *s_sel = reinterpret_cast<uint8_t *>(s_key + L);
+        for (int i = tid; i < L; i += blockDim.x) {
+            const unsigned long long ki = s_key[i];
+            int rank = 0;
+            if (ki != ~0ull) for (int j = 0; j < L; ++j) rank += (s_key[j] < ki) ? 1 : 0;
+            s_sel[i] = (ki != ~0ull && rank < k) ? 1 : 0;
+        }
+        __syncthreads();
+        // its slot in the ascending list is the number of chosen positions before it
+        for (int i = tid; i < L; i += blockDim.x) {
+            if (!s_sel[i]) continue;
+            int slot = 0;
+            for (int j = 0; j < i; ++j) slot += s_sel[j];
+            out[base + slot] = b * S + P + i;
+            if (slot == k - 1) s_last = b * S + P + i;
+        }
+        __syncthreads();
+        const int pad = (k > 0) ? s_last : b * S + P;                  // nothing to choose from: recompute the first response row
+        for (int j = k + tid; j < a.n_adapt; j += blockDim.x) out[base + j] = pad;
+    }
+    if (a.sets_dump) {
+        __syncthreads();
+        for (int j = tid; j < a.n_sel; j += blockDim.x) a.sets_dump[(long long)b * a.n_sel + j] = out[j];
+    }
+}
+
+__global__ void gather_rows_bf16_kernel(const uint4 *__restrict__ src, const int32_t *__restrict__ rows, int chunks, uint4 *__restrict__ dst)
+{
+    const int j = blockIdx.x;
+    const uint4 *s = src + (long long)rows[j] * chunks;
+    uint4 *o = dst + (long long)j * chunks;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) o[c] = s[c];
+}
+
+__global__ void scatter_rows_f32_kernel(const float4 *__restrict__ src, const int32_t *__restrict__ rows, int chunks, float4 *__restrict__ dst)
+{
+    const int j = blockIdx.x;
+    const float4 *s = src + (long long)j * chunks;
+    float4 *o = dst + (long long)rows[j] * chunks;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) o[c] = s[c];
+}
+
+// blockIdx.x = compact row j: copies its K row; blockIdx.y selects a slab of features for the V^T columns
+__global__ void scatter_kv_kernel(const __nv_bfloat16 *__restrict__ qk, long long ld_src, int col0,
+                                  const __nv_bfloat16 *__restrict__ vt_src, long long ld_vt_src, const int32_t *__restrict__ rows,
+                                  int d, __nv_bfloat16 *__restrict__ k_dst, __nv_bfloat16 *__restrict__ vt_dst, long long ld_vt_dst)
+{
+    const int j = blockIdx.x;
+    const int r = rows[j];
+    const uint4 *s = reinterpret_cast<const uint4 *>(qk + (long long)j * ld_src + col0);
+    uint4 *o = reinterpret_cast<uint4 *>(k_dst + (long long)r * d);
+    for (int c = threadIdx.x; c < d / 8; c += blockDim.x) o[c] = s[c];
+    for (int f = threadIdx.x; f < d; f += blockDim.x) vt_dst[(long long)f * ld_vt_dst + r] = vt_src[(long long)f * ld_vt_src + j];
+}
+
+}  // namespace
+
+int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld, int d, int T, float *partial, cudaStream_t s)
+{
+    dim3 grid((unsigned)((T + 63) / 64), kSimSlices, 1);
+    sim_partial_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(vnew_t), reinterpret_cast<const __nv_bfloat16 *>(vold_t),
+                                            ld, d, T, partial);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+int32_t launch_cache_select(const CacheSelectArgs &a, cudaStream_t s)
+{
+    cache_select_kernel<<<a.B, 256, (size_t)a.L * 9 + 16, s>>>(a);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+int32_t launch_gather_rows_bf16(const void *src, const int32_t *rows, int n_rows, int d, void *dst, cudaStream_t s)
+{
+    if (n_rows <= 0) return SFS_OK;
+    gather_rows_bf16_kernel<<<n_rows, 128, 0, s>>>(reinterpret_cast<const uint4 *>(src), rows, d / 8, reinterpret_cast<uint4 *>(dst));
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+int32_t launch_scatter_rows_f32(const float *src, const int32_t *rows, int n_rows, int d, float *dst, cudaStream_t s)
+{
+    if (n_rows <= 0) return SFS_OK;
+    scatter_rows_f32_kernel<<<n_rows, 128, 0, s>>>(reinterpret_cast<const float4 *>(src), rows, d / 4, reinterpret_cast<float4 *>(dst));
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+int32_t launch_scatter_kv(const void *qk_src, long long ld_src, int col0, const void *vt_src, long long ld_vt_src,
+                          const int32_t *rows, int n_rows, int d, void *k_dst, void *vt_dst, long long ld_vt_dst, cudaStream_t s)
+{
+    if (n_rows <= 0) return SFS_OK;
+    scatter_kv_kernel<<<n_rows, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(qk_src), ld_src, col0,
+                                             reinterpret_cast<const __nv_bfloat16 *>(vt_src), ld_vt_src, rows, d,
+                                             reinterpret_cast<__nv_bfloat16 *>(k_dst), reinterpret_cast<__nv_bfloat16 *>(vt_dst), ld_vt_dst);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+}  // namespace sfs

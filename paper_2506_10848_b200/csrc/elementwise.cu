@@ -99,7 +99,7 @@ __global__ void rope_table_kernel(float2 *table, int positions, int half, double
 
 // in place on q and k: pairs (j, j + dh/2) of every head rotate by the angle of the token's position
 __global__ void rope_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int T, int S, int n_heads, int dh,
-                            const float2 *__restrict__ table)
+                            const float2 *__restrict__ table, const int32_t *__restrict__ rows)
 {
     // one thread handles 8 consecutive j of one (token, q-or-k, head)
     const int half = dh / 2, groups = half / 8;
@@ -109,7 +109,7 @@ __global__ void rope_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int T,
     const int g = (int)(idx % groups);
     const int hh = (int)((idx / groups) % (2 * n_heads));      // q heads then k heads: contiguous columns
     const int t = (int)(idx / ((long long)groups * 2 * n_heads));
-    const int pos = t % S;
+    const int pos = (rows ? rows[t] : t) % S;              // compact rows carry the token index they came from
     __nv_bfloat16 *base = qk + (long long)t * ld + (long long)hh * dh + g * 8;
     uint4 lo = *reinterpret_cast<uint4 *>(base), hi = *reinterpret_cast<uint4 *>(base + half);
     const float2 *tb = table + (long long)pos * half + g * 8;
@@ -162,10 +162,10 @@ int32_t launch_rope_table(float2 *table, int positions, int head_dim, float thet
     return SFS_OK;
 }
 
-int32_t launch_rope(void *qk, int64_t ld, int T, int S, int n_heads, int head_dim, const float2 *table, cudaStream_t s)
+int32_t launch_rope(void *qk, int64_t ld, int T, int S, int n_heads, int head_dim, const float2 *table, const int32_t *rows, cudaStream_t s)
 {
     const long long total = (long long)T * 2 * n_heads * (head_dim / 16);
-    rope_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<__nv_bfloat16 *>(qk), ld, T, S, n_heads, head_dim, table);
+    rope_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<__nv_bfloat16 *>(qk), ld, T, S, n_heads, head_dim, table, rows);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }

@@ -4,6 +4,7 @@
 #include "gemm.cuh"
 #include "attention.cuh"
 #include <vector>
+#include <map>
 
 struct sfs_model {
     sfs_config cfg;
@@ -13,6 +14,10 @@ struct sfs_model {
 };
 
 struct LayerPlans { sfs::GemmPlan qkv, o, gate_up, down; };
+// cached mode: per layer, independent of how many rows are recomputed
+struct CacheLayerPlans { sfs::GemmPlan vproj, o_store, down_store; sfs::AttnPlan attn; };
+// cached mode: projections over the compact buffer of recomputed rows, per layer, for one row count
+struct GatherLayerPlans { sfs::GemmPlan qkv, o, gate_up, down; };
 
 struct sfs_session {
     sfs_model *model = nullptr;          // NULL: a selection-only session
@@ -26,7 +31,6 @@ struct sfs_session {
     // forward workspace (model sessions only); T = max_batch*max_seq
     float *x = nullptr;                      // [T, d] fp32 residual stream
     float *partial = nullptr;                // [kMaxSplits, T, d] split-K partial products of the residual projections
-    int pending_partials = 0;                // slabs the next RMSNorm must fold into x
     __nv_bfloat16 *h = nullptr;              // [T, d] normalised activations
     __nv_bfloat16 *qk = nullptr;             // [T, 2d] q | k
     __nv_bfloat16 *vt = nullptr;             // [d, T] V transposed
@@ -48,6 +52,20 @@ struct sfs_session {
     std::vector<LayerPlans> layer_plans;
     sfs::AttnPlan attn_plan;
     sfs::GemmPlan lm_plan;
+    // what the next RMSNorm must fold into x: n slabs `pending_stride` floats apart (split-K partials or a cached increment)
+    const float *pending_ptr = nullptr; int pending_n = 0; long long pending_stride = 0;
+    // feature cache (dLLM-Cache-style), allocated by sfs_cache_enable
+    bool cache_on = false;
+    sfs_cache_params cache_params{};
+    int cache_t = 0, cache_B = 0, cache_S = 0, cache_P = 0;   // step counter and the shape the cached features belong to
+    std::vector<__nv_bfloat16 *> Kc, Vtc;    // per layer: rotated keys [T, d], values transposed [d, T]
+    std::vector<float *> Ac, Fc;             // per layer: residual increments of the attention and MLP branches [T, d]
+    __nv_bfloat16 *hg = nullptr;             // [T, d] gathered normalised rows
+    __nv_bfloat16 *vnew_t = nullptr;         // [d, T] fresh values of every row, transposed
+    float *sim_partial = nullptr;            // [kSimSlices, T, 3]
+    int32_t *sel_rows = nullptr;             // [T] rows recomputed in the current layer
+    std::vector<CacheLayerPlans> cache_plans;
+    std::map<int, std::vector<GatherLayerPlans>> gather_plans;
     // generation bookkeeping (host)
     int32_t gen_B = 0, gen_P = 0, gen_L = 0, gen_cur = 0, gen_steps = 0, gen_max_steps = 0;
     sfs_params gen_params;

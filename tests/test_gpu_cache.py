@@ -1,0 +1,133 @@
+"""GPU parity of the feature cache: cached steps against the oracle's cached forward pass under the SAME schedule
+(the oracle is handed the row sets the GPU chose), the row choice itself against the oracle's rule on the GPU's own
+similarity values (an integer decision: both sides decide on identical numbers), the similarities against the
+oracle's within tolerance, and the cache-off equivalences."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import cache as C
+from oracle import forward as F
+from paper_2506_10848_b200 import binding as sfs
+from paper_2506_10848_b200 import workloads as W
+
+from test_gpu_forward import MAX_ABS, REL_L2, max_abs_bar, tiny_setup
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def state_tensor(B, phase=0, s_cycle=0, hi=0):
+    st = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32)
+    st[:, sfs.STATE_FIELDS.index("phase")] = phase
+    st[:, sfs.STATE_FIELDS.index("s_cycle")] = s_cycle
+    st[:, sfs.STATE_FIELDS.index("hi")] = hi
+    return st.to(DEV)
+
+
+def check_logits(got, ref, scale):
+    err = np.abs(got - ref)
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    assert rel <= REL_L2, rel
+    assert err.max() <= max_abs_bar(scale), err.max()
+
+
+@pytest.mark.parametrize("B,P,L,kp,kr,rho", [(1, 32, 64, 100, 3, 0.25), (2, 24, 40, 4, 2, 0.3), (1, 8, 56, 5, 100, 0.1)])
+def test_cached_steps_match_oracle_under_the_same_schedule(B, P, L, kp, kr, rho):
+    shape, model, cfg, w64 = tiny_setup(seed=3)
+    S = P + L
+    nl = shape.n_layers
+    session = sfs.sfs_session_create(model, B, S)
+    sfs.sfs_cache_enable(session, kp, kr, rho)
+    g = np.random.default_rng(B * 100 + L)
+    tok = np.full((B, S), shape.mask_id, dtype=np.int32)
+    tok[:, :P] = g.integers(0, shape.vocab - 2, size=(B, P))
+    caches = [C.FeatureCache(cfg, S) for _ in range(B)]
+    logits = torch.zeros((B * S, shape.vocab), dtype=torch.float32, device=DEV)
+    sets = torch.full((nl * B * S,), -1, dtype=torch.int32, device=DEV)
+    sims = torch.zeros((nl * B * L,), dtype=torch.float32, device=DEV)
+    n_adapt = C.adaptive_count(rho, L)
+    for step in range(7):
+        if step > 0:                                           # unmask a few positions, as the sampler would
+            for b in range(B):
+                for i in g.choice(L, size=2, replace=False):
+                    tok[b, P + i] = int(g.integers(0, shape.vocab - 2))
+        fast = step in (2, 5)
+        span = (L // 4, L // 4 + 9) if fast else None
+        st = state_tensor(B, 1, span[0], span[1]) if fast else state_tensor(B)
+        d_tok = torch.from_numpy(tok).to(DEV)
+        sets.fill_(-1)
+        n_sel = sfs.sfs_forward_cached(session, d_tok, B, S, P, st, None, None, B * S, logits, sfs.LOGITS_F32, sets=sets, sims=sims)
+        sfs.sfs_check_device_status()
+        rp, rr = step % kp == 0, step % kr == 0
+        assert n_sel == (S if (rp and rr) else (P if rp else 0) + (L if rr else n_adapt))
+        got = logits.cpu().double().numpy().reshape(B, S, -1)
+        gsets = sets.cpu().numpy()[: nl * B * n_sel].reshape(nl, B, n_sel)
+        gsims = sims.cpu().numpy().reshape(nl, B, L)
+        for b in range(B):
+            rec = {}
+            forced = lambda l, s_, c_, b=b: sorted(set(int(r) - b * S - P for r in gsets[l, b] if int(r) - b * S >= P))
+            ref = C.cached_forward(cfg, w64, tok[b], P, caches[b], kp, kr, rho, span=span, select=forced, record=rec)
+            check_logits(got[b], ref, shape.logit_scale)
+            for l in range(nl):
+                # the GPU's sets are exactly the rows of the rule: segment refreshes plus the adaptive choice
+                assert sorted(set(int(r) - b * S for r in gsets[l, b])) == rec["sets"][l], (step, l)
+                if not rr and n_adapt > 0:
+                    cand = list(range(L)) if span is None else list(range(span[0], span[1]))
+                    # integer decision on identical numbers: the oracle's rule applied to the GPU's similarities
+                    mine = C.least_similar(gsims[l, b][cand], cand, min(n_adapt, len(cand)))
+                    chosen = sorted(set(int(r) - b * S - P for r in gsets[l, b] if int(r) - b * S >= P))
+                    assert chosen == mine, (step, l)
+                    # and the similarities themselves agree with the oracle's (bf16 values on the GPU side)
+                    assert np.abs(gsims[l, b][cand] - rec["sims"][l]).max() <= 2e-2, (step, l)
+    sfs.sfs_session_destroy(session)
+    model.close()
+
+
+def test_refresh_every_step_equals_the_uncached_forward_and_unchanged_tokens_do_not_drift():
+    shape, model, cfg, w64 = tiny_setup(seed=4)
+    B, P, L = 1, 16, 48
+    S = P + L
+    session = sfs.sfs_session_create(model, B, S)
+    g = np.random.default_rng(9)
+    tok = np.full((B, S), shape.mask_id, dtype=np.int32)
+    tok[:, :P] = g.integers(0, shape.vocab - 2, size=(B, P))
+    d_tok = torch.from_numpy(tok).to(DEV)
+    plain = torch.zeros((S, shape.vocab), dtype=torch.float32, device=DEV)
+    sfs.sfs_forward(session, d_tok, B, S, None, None, S, plain, sfs.LOGITS_F32)
+    cached = torch.zeros_like(plain)
+    sfs.sfs_cache_enable(session, 1, 1, 0.25)
+    for _ in range(2):
+        sfs.sfs_forward_cached(session, d_tok, B, S, P, None, None, None, S, cached, sfs.LOGITS_F32)
+        # same kernels except that the residual projections store their increments: fp32 rounding order only
+        assert (cached - plain).abs().max().item() <= 2e-3 * shape.logit_scale
+    # any schedule reproduces the same logits while the tokens do not change (cached features are exact then)
+    sfs.sfs_cache_enable(session, 100, 3, 0.2)
+    for step in range(5):
+        sfs.sfs_forward_cached(session, d_tok, B, S, P, None, None, None, S, cached, sfs.LOGITS_F32)
+        assert (cached - plain).abs().max().item() <= 4e-3 * shape.logit_scale, step
+    sfs.sfs_check_device_status()
+    sfs.sfs_session_destroy(session)
+    model.close()
+
+
+def test_generation_with_cache_finishes_and_decodes_every_position_once():
+    shape, model, cfg, w64 = tiny_setup(seed=0, logit_scale=60.0)
+    B, P, L = 2, 32, 64
+    S = P + L
+    session = sfs.sfs_session_create(model, B, S)
+    sfs.sfs_cache_enable(session, 100, 4, 0.25)
+    prompt = W.prompt_ids(B, P, shape.vocab - 2, seed=0).to(DEV)
+    out = torch.zeros((B, S), dtype=torch.int32, device=DEV)
+    state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+    trace = torch.zeros((L + 4, B, sfs.TRACE_INTS), dtype=torch.int32, device=DEV)
+    sfs.sfs_generate(session, prompt, B, P, L, sfs.Params.default(), out, state, trace, L + 4)
+    st = state.cpu().numpy()
+    assert np.all(st[:, sfs.STATE_FIELDS.index("done")] == 1) and np.all(st[:, sfs.STATE_FIELDS.index("n_masked")] == 0)
+    assert np.array_equal(out[:, :P].cpu().numpy(), prompt.cpu().numpy())
+    n_sel = trace[:, :, 5].cpu().numpy()
+    assert np.all(n_sel.sum(axis=0) == L)                                # every position unmasked exactly once
+    sfs.sfs_session_destroy(session)
+    model.close()
