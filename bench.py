@@ -197,12 +197,128 @@ def run_ours(args, rank, world):
                "d2h_bytes_per_step": B * S * 4 / max(gsteps, 1), "steps": gsteps, "seconds": t1 - t0,
                "note": "one sfs_generate call: pinned host prompt -> device, full SlowFast loop, tokens -> pinned host"}
 
-    res = dict(productive=productive, ms=ms, tokens=tokens, launches=launches, clocks=clocks, ms_cls=ms_cls, cnt_cls=cnt_cls, gemm_ms=gemm_ms,
+    extras = None
+    if args.extras and world == 1 and args.workload == "8b" and not args.layers:
+        sfs.sfs_session_destroy(session)
+        session = None
+        torch.cuda.empty_cache()
+        extras = run_extras(torch, sfs, W, model, shape, dev, measured_peaks())
+    res = dict(extras=extras, productive=productive, ms=ms, tokens=tokens, launches=launches, clocks=clocks, ms_cls=ms_cls, cnt_cls=cnt_cls, gemm_ms=gemm_ms,
                gemm_launches=gemm_launches, gemm_tflops=gemm_tflops, prof_steps=prof_steps, e2e=e2e, name=name, shape=shape,
                T=T, S=S, B=B, L=L, P=P, head_rows=head_rows)
-    sfs.sfs_session_destroy(session)
+    if session is not None:
+        sfs.sfs_session_destroy(session)
     model.close()
     return res
+
+
+def time_back_to_back(torch, fn, n):
+    """Device time per call of n calls enqueued back to back (CUDA events on the launching stream)."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / n
+
+
+def run_extras(torch, sfs, W, model, shape, dev, peaks):
+    """The other workloads of the benchmark definition, measured on the same model: the sampling-epilogue
+    microbenchmark, the cached run (prompt 1024 + 512 masked) and the batch of 8 sequences (512 + 256)."""
+    out = {}
+    V = shape.vocab
+    # ---- sampling epilogue: bf16 [256, V] logits with planted winners; 4 rotating copies (259 MB > L2) keep every launch cold
+    R = 256
+    bufs = [W.planted_logits(R, V, seed=1, device=dev) for _ in range(4)]
+    arg = torch.empty(R, dtype=torch.int32, device=dev); sq = torch.empty(R, dtype=torch.int64, device=dev)
+    rs = lambda i: sfs.sfs_row_stats(bufs[i % 4], sfs.LOGITS_BF16, V, V, None, R, argmax=arg, sq=sq)
+    time_back_to_back(torch, rs, 8)
+    us = time_back_to_back(torch, rs, 32) * 1e3
+    # one slow and one fast selection step on those logits (row statistics + transition rule)
+    ssel = sfs.sfs_select_session_create(V, 1, R)
+    rows = torch.arange(R, dtype=torch.int32, device=dev)
+    params = sfs.Params.default()
+    lo, hi = W.span(R, seed=1)
+
+    def sel_step(i, fast):
+        tok = torch.full((1, R), shape.mask_id, dtype=torch.int32, device=dev); msk = torch.ones((1, R), dtype=torch.uint8, device=dev)
+        st = torch.zeros((1, sfs.STATE_INTS), dtype=torch.int32, device=dev)
+        sfs.sfs_state_init(st, 1, R, params)
+        if fast:
+            row = st[0].cpu(); row[sfs.STATE_FIELDS.index("phase")] = 1; row[sfs.STATE_FIELDS.index("s_cycle")] = lo
+            row[sfs.STATE_FIELDS.index("hi")] = hi; st[0] = row.to(dev)
+        cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+        torch.cuda.synchronize()
+        return time_back_to_back(torch, lambda j: sfs.sfs_select(ssel, bufs[(i + j) % 4], sfs.LOGITS_BF16, V, rows, None, R, tok, msk, 1, R, 0, st,
+                                                                  params, sel_count=cnt), 1) * 1e3
+    sel_step(0, False)
+    slow_us, fast_us = sel_step(1, False), sel_step(2, True)
+    sfs.sfs_session_destroy(ssel)
+    gbs = R * V * 2 / us * 1e-3
+    out["epilogue"] = {"workload": f"bf16 logits [{R}, {V}], planted winners, seed 1; cold (4 rotating copies > L2)", "row_stats_us": us,
+                       "hbm_gbs": gbs, "frac_of_measured_hbm_peak": gbs / peaks["hbm_gbs"], "select_slow_step_us": slow_us,
+                       "select_fast_step_us": fast_us, "span": [lo, hi]}
+    del bufs
+    torch.cuda.empty_cache()
+
+    def timed_steps(session, n):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        evs[0].record()
+        for i in range(n):
+            sfs.sfs_generate_steps(session, 1, None, 0)
+            evs[i + 1].record()
+        torch.cuda.synchronize()
+        return [evs[i].elapsed_time(evs[i + 1]) for i in range(n)]
+
+    # ---- prompt 1024 + 512 masked, feature cache on (K_p 100, K_r 5, rho 0.25) against off
+    B, P, L = 1, 1024, 512
+    session = sfs.sfs_session_create(model, B, P + L)
+    prompt = W.prompt_ids(B, P, V - 2, seed=3).to(dev)
+    sfs.sfs_generate_begin(session, prompt, B, P, L, params)
+    timed_steps(session, 2)
+    plain = timed_steps(session, 5)
+    sfs.sfs_cache_enable(session, 100, 5, 0.25)
+    sfs.sfs_generate_begin(session, prompt, B, P, L, params)
+    cached = timed_steps(session, 11)                       # steps 0..10: full refresh at 0, response refresh at 5 and 10
+    sfs.sfs_check_device_status()
+    part = [cached[i] for i in (1, 2, 3, 4, 6, 7, 8, 9)]
+    out["cached_1024_512"] = {"workload": "8B shape, batch 1, prompt 1024 + 512 masked, seed 3", "uncached_ms_per_step": sum(plain) / len(plain),
+                              "cached_ms_per_step_cycle_avg": sum(cached[1:6]) / 5, "cached_partial_step_ms": sum(part) / len(part),
+                              "cached_response_refresh_step_ms": (cached[5] + cached[10]) / 2, "cached_full_refresh_step_ms": cached[0],
+                              "params": "K_p 100, K_r 5, rho 0.25"}
+    out["cached_1024_512"]["speedup"] = out["cached_1024_512"]["uncached_ms_per_step"] / out["cached_1024_512"]["cached_ms_per_step_cycle_avg"]
+    sfs.sfs_session_destroy(session)
+    torch.cuda.empty_cache()
+
+    # ---- batch of 8 independent sequences, prompt 512 + 256 masked
+    B, P, L = 8, 512, 256
+    session = sfs.sfs_session_create(model, B, P + L)
+    prompt = W.prompt_ids(B, P, V - 2, seed=4).to(dev)
+    sfs.sfs_generate_begin(session, prompt, B, P, L, params)
+    timed_steps(session, 2)
+    ts = timed_steps(session, 6)
+    sfs.sfs_check_device_status()
+    ms = sum(ts) / len(ts)
+    g_fl, a_fl, h_fl = step_flops(shape, B * (P + L), P + L, B * L)
+    roof = max((g_fl + a_fl + h_fl) / (peaks["bf16_tflops"] * 1e12), step_bytes(shape, B * (P + L), B * L) / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    out["batch8_512_256"] = {"workload": "8B shape, batch 8, prompt 512 + 256 masked, seed 4", "ms_per_step": ms, "tokens_per_s": B / (ms * 1e-3),
+                             "step_roofline_ms": roof, "step_roofline_frac": roof / ms,
+                             "note": "one token per sequence and step with random-init logits"}
+    sfs.sfs_session_destroy(session)
+    torch.cuda.empty_cache()
+    return out
+
+
+def aggregate(torch, ms, tokens, launches, world, device):
+    """Whole-job numbers over the ranks: slowest rank's time, summed tokens and launches."""
+    if world <= 1:
+        return ms, tokens, launches
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    k = torch.tensor([tokens, launches], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(k, op=torch.distributed.ReduceOp.SUM)
+    return float(t[0]), int(k[0]), int(k[1])
 
 
 def oracle_sample(shape, P, L, seed=2):
@@ -273,6 +389,7 @@ def main():
     ap.add_argument("--workload", default="8b", choices=["8b", "tiny"])
     ap.add_argument("--layers", type=int, default=0, help="keep only this many layers (small case for ncu captures)")
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")
+    ap.add_argument("--no-extras", dest="extras", action="store_false", help="skip the epilogue / cached / batch-8 workloads")
     ap.add_argument("--no-cpu-baseline", dest="cpu", action="store_false")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
@@ -295,14 +412,7 @@ def main():
     res = run_ours(args, rank, world)
 
     ms, tokens = res["ms"], res["tokens"]
-    if world > 1:
-        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        k = torch.tensor([tokens, res["launches"]], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(k, op=torch.distributed.ReduceOp.SUM)
-        ms, tokens, launches = float(t[0]), int(k[0]), int(k[1])
-    else:
-        launches = res["launches"]
+    ms, tokens, launches = aggregate(torch, ms, tokens, res["launches"], world, "cuda")
     if rank != 0:
         if world > 1:
             torch.distributed.destroy_process_group()
@@ -328,6 +438,8 @@ def main():
             "step_roofline_ms": step_roof_ms, "step_roofline_frac": step_roof_ms / ms_step,
             "kernel_ms_per_step": {k: v / res["prof_steps"] for k, v in res["ms_cls"].items()},
             "roofline": roofline, "e2e": res["e2e"]}
+    if res["extras"]:
+        line.update(res["extras"])
     if args.cpu and world == 1:
         from paper_2506_10848_b200 import workloads as W
         P, L = (32, 64) if args.workload == "tiny" else (256, 256)

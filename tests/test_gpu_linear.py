@@ -42,3 +42,16 @@ def test_linear_wide_tile_config():
     # enough tiles that the 128 x 256 configuration is chosen
     got, ref = run(1024, 8192, 512, 1, seed=3)
     assert np.abs(got - ref).max() <= 1e-3 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("M,N,K,out_dtype", [(512, 12288, 4096, 1), (512, 12288, 4096, 0), (384, 6144, 2048, 1), (512, 3000, 1024, 0)])
+def test_linear_few_wide_tiles(M, N, K, out_dtype):
+    """Shapes with fewer wide tiles than SM pairs (the planner narrows the tiles), large K, ragged N; bf16 and fp32 out."""
+    for rep in range(2):
+        got, ref = run(M, N, K, out_dtype, seed=5 + rep)
+        if out_dtype:
+            assert np.abs(got - ref).max() <= 1e-3 * np.abs(ref).max()
+        else:
+            # one bf16 rounding (half an ulp: up to 2^-8 relative) of an fp32 sum of K products whose own error grows with K
+            rel = np.abs(got - ref) / np.maximum(np.abs(ref), 1.0)
+            assert rel.max() <= 2.0 ** -8 + 1e-7 * K
