@@ -112,7 +112,7 @@ constexpr uint32_t kNegInf2 = 0xFF80FF80u;
 
 // One cluster (1, 2, 4 or 8 CTAs) per logits row; NV 16-byte chunks per thread.
 template <int NV>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 4)
 rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int nchunks, int vocab,
                       const int32_t *__restrict__ n_rows_ptr, int max_rows, RowOut out)
 {
