@@ -3,8 +3,9 @@
 //
 // One CTA owns 128 query rows of one (sequence, head).  Warp 0 streams K tiles [128 keys x dh] and V^T
 // tiles [dh x 128 keys] through a two-stage TMA ring, warp 1 issues tcgen05.mma for S = Q K^T (accumulator
-// in tensor memory) and for O_j = P V_j, warps 2-5 (one thread per query row) run the online softmax in fp32
-// on S read back with tcgen05.ld, write P as bf16 into shared memory in the 128-byte-swizzled K-major
+// in tensor memory) and for O_j = P V_j, warps 2-9 (two threads per query row: each takes half of a tile's keys and
+// half of the output columns, so two warps share a scheduler and hide each other's latencies) run the online softmax
+// in fp32 on S read back with tcgen05.ld, write P as bf16 into shared memory in the 128-byte-swizzled K-major
 // layout the next MMA consumes, and fold each O_j into a register accumulator with the running rescale.
 // V is consumed transposed (features x tokens); the QKV projection's epilogue writes it that way.
 #include "sfs_common.cuh"
@@ -14,7 +15,7 @@
 namespace sfs {
 namespace {
 
-constexpr int kAttnThreads = 192;
+constexpr int kAttnThreads = 64 + 256;   // TMA warp, MMA warp, 8 softmax warps
 constexpr int QT = 128;                 // query rows per CTA
 constexpr int KT = 128;                 // keys per tile
 constexpr int KV_STAGES = 2;
@@ -36,8 +37,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = smem, *sKV = smem + Q_BYTES, *sP = sKV + KV_STAGES * STAGE_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(sP + P_BYTES);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * KV_STAGES + 4);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * KV_STAGES + 5);
     __shared__ int s_abort;
+    __shared__ float s_xch[2][2][QT];                      // [tile parity][key half][row]: maxima (denominators at the end)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int q0 = blockIdx.x * QT, h = blockIdx.y, b = blockIdx.z;
@@ -47,11 +49,11 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int nkv = (S + KT - 1) / KT;
 
     const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * KV_STAGES;
-    const uint32_t bar_q = bar_empty + 8 * KV_STAGES, bar_s = bar_q + 8, bar_p = bar_q + 16, bar_o = bar_q + 24;
+    const uint32_t bar_q = bar_empty + 8 * KV_STAGES, bar_s = bar_q + 8, bar_p = bar_q + 16, bar_o = bar_q + 24, bar_x = bar_q + 32;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < KV_STAGES; ++s) { tc::mbar_init(bar_full + 8 * s, 1); tc::mbar_init(bar_empty + 8 * s, 1); }
-        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_s, 1); tc::mbar_init(bar_p, 128); tc::mbar_init(bar_o, 1);
+        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_s, 1); tc::mbar_init(bar_p, 256); tc::mbar_init(bar_o, 1); tc::mbar_init(bar_x, 256);
         s_abort = 0;
         tc::mbar_init_fence();
     }
@@ -141,54 +143,57 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
     } else {
-        // ---------------- online softmax + output accumulation: thread = query row
-        const int qd = warp & 3;
+        // ---------------- online softmax + output accumulation: two threads per query row
+        constexpr int HK = KT / 2;                         // keys of a tile per thread
+        constexpr int HD = DH / 2;                         // output columns per thread
+        const int qd = warp & 3, half = (warp - 2) >> 2;
         const int row = qd * 32 + lane;
         const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
         const float c = a.scale_log2;                      // log2(e) / sqrt(dh)
-        float m = -INFINITY, l = 0.f;
-        float acc[DH];
+        float m = -INFINITY, l = 0.f;                      // l: this thread's keys only; the halves are added at the end
+        float acc[HD];
 #pragma unroll
-        for (int i = 0; i < DH; ++i) acc[i] = 0.f;
+        for (int i = 0; i < HD; ++i) acc[i] = 0.f;
         bool ok = true;
         for (int j = 0; j < nkv && ok; ++j) {
             ok = tc::mbar_wait(bar_s, (uint32_t)j & 1u, &s_abort);
             if (!ok) break;
             tc::tc_fence_after();
-            const int valid = min(KT, S - j * KT);         // keys of this tile that belong to the sequence
+            const int valid = min(KT, S - j * KT) - half * HK;     // keys of this thread's half that belong to the sequence
+            uint32_t v[HK];
+#pragma unroll
+            for (int cc = 0; cc < HK / 32; ++cc) tc::tmem_ld32(tmem_S + lane_off + half * HK + cc * 32, v + cc * 32);
+            tc::tmem_ld_wait();
             float mx = -INFINITY;
 #pragma unroll
-            for (int cc = 0; cc < KT / 32; ++cc) {
-                uint32_t v[32];
-                tc::tmem_ld32(tmem_S + lane_off + cc * 32, v);
-                tc::tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (cc * 32 + i < valid) mx = fmaxf(mx, __uint_as_float(v[i]));
-            }
-            const float m_new = fmaxf(m, mx);
+            for (int i = 0; i < HK; ++i)
+                if (i < valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+            s_xch[j & 1][half][row] = mx;                  // exchange the two halves' maxima (bounded wait, like every other)
+            tc::mbar_arrive(bar_x);
+            ok = tc::mbar_wait(bar_x, (uint32_t)j & 1u, &s_abort);
+            if (!ok) break;
+            const float m_new = fmaxf(m, fmaxf(mx, s_xch[j & 1][half ^ 1][row]));
             const float alpha = exp2f((m - m_new) * c);
             const float mc = m_new * c;
             float lsum = 0.f;
 #pragma unroll
-            for (int cc = 0; cc < KT / 32; ++cc) {
-                uint32_t v[32];
-                tc::tmem_ld32(tmem_S + lane_off + cc * 32, v);
-                tc::tmem_ld_wait();
+            for (int cc = 0; cc < HK / 32; ++cc) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float p0 = (cc * 32 + 2 * i < valid) ? exp2f(fmaf(__uint_as_float(v[2 * i]), c, -mc)) : 0.f;
-                    const float p1 = (cc * 32 + 2 * i + 1 < valid) ? exp2f(fmaf(__uint_as_float(v[2 * i + 1]), c, -mc)) : 0.f;
+                    const float p0 = (cc * 32 + 2 * i < valid) ? exp2f(fmaf(__uint_as_float(v[cc * 32 + 2 * i]), c, -mc)) : 0.f;
+                    const float p1 = (cc * 32 + 2 * i + 1 < valid) ? exp2f(fmaf(__uint_as_float(v[cc * 32 + 2 * i + 1]), c, -mc)) : 0.f;
                     lsum += p0 + p1;
                     __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     pk[i] = *reinterpret_cast<uint32_t *>(&hh);
                 }
-                // keys cc*32 .. cc*32+31 of this row: K-block cc/2, 16-byte chunks (cc%2)*4 .. +3, swizzled by row
-                uint8_t *prow = sP + (cc >> 1) * (QT * 128) + row * 128;
+                // keys kc*32 .. kc*32+31 of this row (kc counts 32-key groups of the tile): K-block kc/2, 16-byte chunks
+                // (kc%2)*4 .. +3, swizzled by row
+                const int kc = half * (HK / 32) + cc;
+                uint8_t *prow = sP + (kc >> 1) * (QT * 128) + row * 128;
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4) {
-                    const int chunk = ((cc & 1) * 4 + q4) ^ (row & 7);
+                    const int chunk = ((kc & 1) * 4 + q4) ^ (row & 7);
                     *reinterpret_cast<uint4 *>(prow + chunk * 16) = make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
                 }
             }
@@ -201,20 +206,24 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             if (!ok) break;
             tc::tc_fence_after();
 #pragma unroll
-            for (int cc = 0; cc < DH / 32; ++cc) {
-                uint32_t v[32];
-                tc::tmem_ld32(tmem_O + lane_off + cc * 32, v);
+            for (int cc = 0; cc < HD / 32; ++cc) {
+                uint32_t o[32];
+                tc::tmem_ld32(tmem_O + lane_off + half * HD + cc * 32, o);
                 tc::tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[cc * 32 + i] = fmaf(acc[cc * 32 + i], alpha, __uint_as_float(v[i]));
+                for (int i = 0; i < 32; ++i) acc[cc * 32 + i] = fmaf(acc[cc * 32 + i], alpha, __uint_as_float(o[i]));
             }
             tc::tc_fence_before();
         }
+        // the two halves of a row add their partial denominators
+        s_xch[nkv & 1][half][row] = l;
+        tc::mbar_arrive(bar_x);
+        ok = ok && tc::mbar_wait(bar_x, (uint32_t)nkv & 1u, &s_abort);
         if (ok && !s_abort && q0 + row < a.kq) {
-            const float inv = 1.0f / l;
-            __nv_bfloat16 *dst = a.out + (long long)(qrow0 + row) * a.ld_out + h * DH;
+            const float inv = 1.0f / (l + s_xch[nkv & 1][half ^ 1][row]);
+            __nv_bfloat16 *dst = a.out + (long long)(qrow0 + row) * a.ld_out + h * DH + half * HD;
 #pragma unroll
-            for (int i = 0; i < DH / 8; ++i) {
+            for (int i = 0; i < HD / 8; ++i) {
                 uint32_t o[4];
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
@@ -236,7 +245,7 @@ template <int DH>
 int32_t launch_dh(const AttnPlan &p, int kq, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
     constexpr size_t smem = (size_t)QT * DH * 2 + KV_STAGES * (size_t)(KT * DH * 2 + DH * KT * 2) + QT * KT * 2
-                          + (2 * KV_STAGES + 4) * 8 + 16 + 1024;
+                          + (2 * KV_STAGES + 5) * 8 + 16 + 1024;
     static bool configured = false;
     if (!configured) {
         SFS_CUDA(cudaFuncSetAttribute(attention_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
