@@ -37,15 +37,17 @@ static int32_t check_params(const sfs_params *p)
 }
 
 // one sticky device status word per process (set by kernels whose bounded waits give up)
+static int32_t *g_status_word = nullptr;
 int32_t *device_status_word()
 {
-    static int32_t *w = nullptr;
-    if (!w) {
-        if (cudaMalloc(&w, 256) != cudaSuccess) { w = nullptr; return nullptr; }
-        cudaMemset(w, 0, 256);
+    if (!g_status_word) {
+        if (cudaMalloc(&g_status_word, 256) != cudaSuccess) { g_status_word = nullptr; return nullptr; }
+        cudaMemset(g_status_word, 0, 256);
     }
-    return w;
+    return g_status_word;
 }
+// the word if some earlier call has created it, else null: never allocates
+int32_t *device_status_word_if_any() { return g_status_word; }
 
 template <typename T>
 static int32_t dev_alloc(sfs_session *s, T **out, size_t count, bool zero)

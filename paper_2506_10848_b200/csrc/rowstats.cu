@@ -14,6 +14,7 @@
 namespace cg = cooperative_groups;
 
 namespace sfs {
+int32_t *device_status_word_if_any();     // the process's sticky status word, null until some call has created it
 namespace {
 
 constexpr float kLog2e = 0x1.715476p+0f;
@@ -114,7 +115,7 @@ constexpr uint32_t kNegInf2 = 0xFF80FF80u;
 template <int NV>
 __global__ void __launch_bounds__(kThreads, 4)
 rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int nchunks, int vocab,
-                      const int32_t *__restrict__ n_rows_ptr, int max_rows, RowOut out)
+                      const int32_t *__restrict__ n_rows_ptr, int max_rows, RowOut out, int32_t *err)
 {
     cg::cluster_group cluster = cg::this_cluster();
     const int C    = (int)cluster.num_blocks();
@@ -125,8 +126,9 @@ rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int
 
     __shared__ float s_wmax[kThreads / 32];
     __shared__ unsigned long long s_wsum[kThreads / 32];
-    __shared__ float s_cta_max;
-    __shared__ unsigned long long s_cta_sum;
+    __shared__ float s_max_of[8];                           // slice maxima of all CTAs of the cluster, pushed by their owners
+    __shared__ unsigned long long s_row_sum;                // rank 0 only: the peers add their sums here ...
+    __shared__ int s_row_arg, s_arrived;                    // ... and their first-maximum candidates, then count themselves in
     __shared__ int s_cta_arg;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -139,7 +141,7 @@ rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int
         const int chunk = (j * C + rank) * kThreads + tid;
         v[j] = (chunk < nchunks) ? ld_stream(rp + chunk) : make_uint4(kNegInf2, kNegInf2, kNegInf2, kNegInf2);
     }
-    if (tid == 0) s_cta_arg = 0x7FFFFFFF;
+    if (tid == 0) { s_cta_arg = 0x7FFFFFFF; s_row_sum = 0; s_row_arg = 0x7FFFFFFF; s_arrived = 0; }
 
     // ---- pass 1: exact maximum
     __nv_bfloat162 mx = as_bf162(kNegInf2);
@@ -151,19 +153,22 @@ rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int
     float m = warp_max(lmax);
     if (lane == 0) s_wmax[warp] = m;
     __syncthreads();
-    if (tid == 0) {
-        float t = s_wmax[0];
-#pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) t = fmaxf(t, s_wmax[w]);
-        s_cta_max = t;
-    }
     if (C > 1) {
+        // every CTA pushes its slice maximum into every CTA's table; after the one cluster barrier nobody reads a peer's
+        // shared memory any more (only rank 0's is written to, and rank 0 stays until everybody has reported)
+        if (tid < C) {
+            float t = s_wmax[0];
+#pragma unroll
+            for (int w = 1; w < kThreads / 32; ++w) t = fmaxf(t, s_wmax[w]);
+            *cluster.map_shared_rank(&s_max_of[rank], tid) = t;
+        }
         cluster.sync();
-        m = -INFINITY;
-        for (int r = 0; r < C; ++r) m = fmaxf(m, *cluster.map_shared_rank(&s_cta_max, r));
+        m = s_max_of[0];
+        for (int r = 1; r < C; ++r) m = fmaxf(m, s_max_of[r]);
     } else {
-        __syncthreads();
-        m = s_cta_max;
+        m = s_wmax[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) m = fmaxf(m, s_wmax[w]);
     }
 
     // ---- first position of the maximum (only threads that hold it look)
@@ -203,22 +208,26 @@ rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int
         unsigned long long t = 0;
 #pragma unroll
         for (int w = 0; w < kThreads / 32; ++w) t += s_wsum[w];
-        s_cta_sum = t;
-    }
-    if (C > 1) {
-        cluster.sync();                                     // sums and argmin candidates of all CTAs are visible
-        if (rank == 0 && tid == 0) {
-            unsigned long long S = 0; int arg = 0x7FFFFFFF;
-            for (int r = 0; r < C; ++r) {
-                S += *cluster.map_shared_rank(&s_cta_sum, r);
-                arg = min(arg, *cluster.map_shared_rank(&s_cta_arg, r));
+        const int arg = s_cta_arg;
+        if (C > 1) {
+            // report to rank 0 (integer adds and a minimum: any arrival order gives the same result), then leave
+            unsigned long long *rs = cluster.map_shared_rank(&s_row_sum, 0);
+            int *ra = cluster.map_shared_rank(&s_row_arg, 0), *rn = cluster.map_shared_rank(&s_arrived, 0);
+            atomicAdd(rs, t);
+            atomicMin(ra, arg);
+            __threadfence();
+            atomicAdd(rn, 1);
+            if (rank == 0) {
+                int spins = 0;
+                while (*reinterpret_cast<volatile int *>(&s_arrived) < C && ++spins < (1 << 24)) {}
+                if (spins >= (1 << 24) && err) atomicExch(err, SFS_ERR_TIMEOUT);   // a peer never reported
+                __threadfence();
+                const int a2 = *reinterpret_cast<volatile int *>(&s_row_arg);
+                write_row(out, row, a2 == 0x7FFFFFFF ? 0 : a2, *reinterpret_cast<volatile unsigned long long *>(&s_row_sum));
             }
-            write_row(out, row, arg == 0x7FFFFFFF ? 0 : arg, S);
+        } else {
+            write_row(out, row, arg == 0x7FFFFFFF ? 0 : arg, t);
         }
-        cluster.sync();                                     // keep remote shared memory alive until rank 0 has read it
-    } else {
-        __syncthreads();
-        if (tid == 0) write_row(out, row, s_cta_arg == 0x7FFFFFFF ? 0 : s_cta_arg, s_cta_sum);
     }
 }
 
@@ -288,7 +297,8 @@ int32_t launch_cluster(const uint4 *logits, long long ld_chunks, int nchunks, in
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_cluster_bf16<NV>, logits, ld_chunks, nchunks, vocab, d_n_rows, max_rows, out));
+    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_cluster_bf16<NV>, logits, ld_chunks, nchunks, vocab, d_n_rows, max_rows, out,
+                                device_status_word_if_any()));
     return SFS_OK;
 }
 
