@@ -123,3 +123,72 @@ def test_batch_of_eight_is_eight_independent_sequences(model8b):
         assert np.all((o[:, P:] != shape.mask_id).sum(dim=1).numpy() >= unmasked - 1)   # (an argmax may be the mask id itself)
     finally:
         sfs.sfs_session_destroy(session)
+
+
+def test_cached_steps_match_the_oracle_at_the_8b_shape_under_the_same_schedule(model8b):
+    """Prompt 1024 + 512 masked with the feature cache: one refresh step, one slow partial step and one fast partial step
+    (candidates = the span).  The oracle runs the same schedule in fp32 and is handed the rows the GPU chose; the row
+    choice itself is checked against the oracle's rule applied to the GPU's own similarities (an integer decision)."""
+    from oracle import cache as C
+    shape, w, model = model8b
+    B, P, L = 1, 1024, 512
+    S = P + L
+    nl = shape.n_layers
+    kp, kr, rho = 100, 8, 0.25
+    g = np.random.default_rng(3)
+    tok = np.full((B, S), shape.mask_id, dtype=np.int32)
+    tok[:, :P] = W.prompt_ids(B, P, shape.vocab - 2, seed=3).numpy()
+    conv = lambda t: t.detach().to("cpu").to(torch.float32).numpy()
+    w_or = {"tok_emb": conv(w["tok_emb"]), "final_norm": conv(w["final_norm"]), "lm_head": conv(w["lm_head"]), "layers": LazyLayers(w["layers"])}
+    cfg = F.ModelConfig(**shape.asdict())
+    cache = C.FeatureCache(cfg, S, dtype=np.float32)
+    rows = [P, P + 1, P + 130, P + 255, S - 1, 17]
+    n_adapt = C.adaptive_count(rho, L)
+    span = (120, 200)
+    session = sfs.sfs_session_create(model, B, S)
+    try:
+        sfs.sfs_cache_enable(session, kp, kr, rho)
+        d_rows = torch.tensor(rows, dtype=torch.int32, device=DEV)
+        lg = torch.zeros((len(rows), shape.vocab), dtype=torch.float32, device=DEV)
+        sets = torch.full((nl * B * S,), -1, dtype=torch.int32, device=DEV)
+        sims = torch.zeros((nl * B * L,), dtype=torch.float32, device=DEV)
+        st = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32)
+        for step in range(3):
+            if step > 0:
+                for i in g.choice(L, size=4, replace=False):
+                    tok[0, P + i] = int(g.integers(0, shape.vocab - 2))
+            fast = step == 2
+            st.zero_()
+            if fast:
+                st[:, sfs.STATE_FIELDS.index("phase")] = 1
+                st[:, sfs.STATE_FIELDS.index("s_cycle")] = span[0]
+                st[:, sfs.STATE_FIELDS.index("hi")] = span[1]
+            sets.fill_(-1)
+            n_sel = sfs.sfs_forward_cached(session, torch.from_numpy(tok).to(DEV), B, S, P, st.to(DEV), d_rows, None, len(rows), lg,
+                                           sfs.LOGITS_F32, sets=sets, sims=sims)
+            sfs.sfs_check_device_status()
+            assert n_sel == (S if step == 0 else n_adapt)          # fixed-size list: a short span is padded by repetition
+            got = lg.cpu().double().numpy()
+            gsets = sets.cpu().numpy()[: nl * n_sel].reshape(nl, n_sel)
+            gsims = sims.cpu().numpy().reshape(nl, L)
+            rec = {}
+            forced = lambda l, s_, c_: sorted(set(int(r) - P for r in gsets[l] if int(r) >= P))
+            ref = C.cached_forward(cfg, w_or, tok[0], P, cache, kp, kr, rho, span=span if fast else None, rows=rows,
+                                   select=forced, record=rec).astype(np.float64)
+            rel_l2 = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+            max_abs = np.abs(got - ref).max()
+            tol_rel, tol_abs = tolerances(nl, ref)
+            worst_sim = 0.0
+            for l in range(nl):
+                assert sorted(set(int(r) for r in gsets[l])) == rec["sets"][l], (step, l)
+                if step > 0:
+                    cand = list(range(L)) if not fast else list(range(span[0], span[1]))
+                    mine = C.least_similar(gsims[l][cand], cand, min(n_adapt, len(cand)))
+                    assert sorted(set(int(r) - P for r in gsets[l])) == mine, (step, l)
+                    worst_sim = max(worst_sim, float(np.abs(gsims[l][cand] - rec["sims"][l]).max()))
+            print(f"8B cached step {step}: n_sel={n_sel} max_abs={max_abs:.4g} rel_l2={rel_l2:.4g} sims diff {worst_sim:.3g}")
+            assert rel_l2 <= tol_rel and max_abs <= tol_abs, (step, rel_l2, tol_rel, max_abs, tol_abs)
+            assert worst_sim <= 5e-2, (step, worst_sim)
+    finally:
+        sfs.sfs_cache_enable(session, 1, 1, 0.0, off=True)
+        sfs.sfs_session_destroy(session)
