@@ -1,13 +1,15 @@
 // Bidirectional (unmasked) multi-head attention of the mask predictor: out = softmax(q k^T / sqrt(dh)) v
 // over all S positions of the same sequence.
 //
-// One CTA owns 128 query rows of one (sequence, head).  Warp 0 streams K tiles [128 keys x dh] and V^T
-// tiles [dh x 128 keys] through a two-stage TMA ring, warp 1 issues tcgen05.mma for S = Q K^T (accumulator
-// in tensor memory) and for O_j = P V_j, warps 2-9 (two threads per query row: each takes half of a tile's keys and
-// half of the output columns, so two warps share a scheduler and hide each other's latencies) run the online softmax
-// in fp32 on S read back with tcgen05.ld, write P as bf16 into shared memory in the 128-byte-swizzled K-major
-// layout the next MMA consumes, and fold each O_j into a register accumulator with the running rescale.
-// V is consumed transposed (features x tokens); the QKV projection's epilogue writes it that way.
+// One CTA owns 128 query rows of one (sequence, head).  Warp 0 streams K tiles [128 keys x dh] and V^T tiles
+// [dh x 128 keys] through two two-stage TMA rings.  Warp 1 issues tcgen05.mma: S_j = Q K_j^T into one of two score
+// buffers in tensor memory, and O += P_j V_j into an accumulator that stays in tensor memory for the whole row of tiles;
+// S_{j+1} is issued before P_j V_j, so the tensor core computes the next scores while the softmax runs.  Warps 2-9 (two
+// threads per query row: each takes half of a tile's keys and half of the output columns) read S back with tcgen05.ld,
+// run the online softmax in fp32 and write P as bf16 into shared memory in the 128-byte-swizzled K-major layout the
+// next MMA consumes.  The exponentials use a reference maximum that is moved (with a rescale of O and of the denominator)
+// only when the true running maximum has outgrown it by 2^8: the result is the same softmax, most tiles skip the pass
+// over O.  V is consumed transposed (features x tokens); the QKV projection's epilogue writes it that way.
 #include "sfs_common.cuh"
 #include "tc05.cuh"
 #include "attention.cuh"
@@ -19,6 +21,7 @@ constexpr int kAttnThreads = 64 + 256;   // TMA warp, MMA warp, 8 softmax warps
 constexpr int QT = 128;                 // query rows per CTA
 constexpr int KT = 128;                 // keys per tile
 constexpr int KV_STAGES = 2;
+constexpr int kAttnBars = 4 * KV_STAGES + 6;   // K full/empty, V full/empty, Q, S (two), P, O, exchange
 
 template <int DH>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -29,15 +32,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     constexpr int K_BYTES = KT * DH * 2;
     constexpr int V_BYTES = DH * KT * 2;
     constexpr int P_BYTES = QT * KT * 2;
-    constexpr int STAGE_BYTES = K_BYTES + V_BYTES;
-    constexpr uint32_t TMEM_COLS = (KT + DH) <= 256 ? 256 : 512;
+    constexpr uint32_t TMEM_COLS = 512;                  // S (two buffers of 128 columns) and O (DH columns)
 
     if (a.d_active && *a.d_active == 0) return;          // nothing left to decode: uniform early exit
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t *sQ = smem, *sKV = smem + Q_BYTES, *sP = sKV + KV_STAGES * STAGE_BYTES;
+    uint8_t *sQ = smem, *sK = smem + Q_BYTES, *sV = sK + KV_STAGES * K_BYTES, *sP = sV + KV_STAGES * V_BYTES;
     uint64_t *bars = reinterpret_cast<uint64_t *>(sP + P_BYTES);
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * KV_STAGES + 5);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + kAttnBars);
     __shared__ int s_abort;
     __shared__ float s_xch[2][2][QT];                      // [tile parity][key half][row]: maxima (denominators at the end)
 
@@ -48,12 +50,17 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const int qrow0 = b * a.kq + q0;                       // first query row of this CTA (queries may be a compact subset)
     const int nkv = (S + KT - 1) / KT;
 
-    const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * KV_STAGES;
-    const uint32_t bar_q = bar_empty + 8 * KV_STAGES, bar_s = bar_q + 8, bar_p = bar_q + 16, bar_o = bar_q + 24, bar_x = bar_q + 32;
+    const uint32_t bar_kfull = tc::smem_u32(bars), bar_kempty = bar_kfull + 8 * KV_STAGES;
+    const uint32_t bar_vfull = bar_kempty + 8 * KV_STAGES, bar_vempty = bar_vfull + 8 * KV_STAGES;
+    const uint32_t bar_q = bar_vempty + 8 * KV_STAGES, bar_s = bar_q + 8 /* two */, bar_p = bar_q + 24, bar_o = bar_q + 32, bar_x = bar_q + 40;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < KV_STAGES; ++s) { tc::mbar_init(bar_full + 8 * s, 1); tc::mbar_init(bar_empty + 8 * s, 1); }
-        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_s, 1); tc::mbar_init(bar_p, 256); tc::mbar_init(bar_o, 1); tc::mbar_init(bar_x, 256);
+        for (int s = 0; s < KV_STAGES; ++s) {
+            tc::mbar_init(bar_kfull + 8 * s, 1); tc::mbar_init(bar_kempty + 8 * s, 1);
+            tc::mbar_init(bar_vfull + 8 * s, 1); tc::mbar_init(bar_vempty + 8 * s, 1);
+        }
+        tc::mbar_init(bar_q, 1); tc::mbar_init(bar_s, 1); tc::mbar_init(bar_s + 8, 1);
+        tc::mbar_init(bar_p, 256); tc::mbar_init(bar_o, 1); tc::mbar_init(bar_x, 256);
         s_abort = 0;
         tc::mbar_init_fence();
     }
@@ -62,128 +69,171 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
-    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + KT;
+    const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 2 * KT;
 
     if (warp == 0) {
         if (lane == 0) {
-            // ---------------- TMA producer: Q once, then K / V^T tiles
+            // ---------------- TMA producer: Q once, then K tiles and V^T tiles through their own rings (a K stage is free
+            // again as soon as its S = Q K^T has been computed, a V stage after its P V)
             tc::mbar_expect_tx(bar_q, Q_BYTES);
 #pragma unroll
             for (int kb = 0; kb < KB; ++kb)
                 tc::tma_load_2d(tc::smem_u32(sQ) + kb * (QT * 128), &tmQ, h * DH + kb * 64, qrow0, bar_q);
-            int issued = 0;
+            int issued_k = 0, issued_v = 0;
             for (int j = 0; j < nkv; ++j) {
                 const int s = j % KV_STAGES;
                 const uint32_t ph = (uint32_t)(j / KV_STAGES) & 1u;
-                if (!tc::mbar_wait(bar_empty + 8 * s, ph ^ 1u, &s_abort)) break;
-                const uint32_t sk = tc::smem_u32(sKV) + s * STAGE_BYTES, sv = sk + K_BYTES;
-                tc::mbar_expect_tx(bar_full + 8 * s, STAGE_BYTES);
+                if (!tc::mbar_wait(bar_kempty + 8 * s, ph ^ 1u, &s_abort)) break;
+                const uint32_t sk = tc::smem_u32(sK) + s * K_BYTES;
+                tc::mbar_expect_tx(bar_kfull + 8 * s, K_BYTES);
 #pragma unroll
                 for (int kb = 0; kb < KB; ++kb)
-                    tc::tma_load_2d(sk + kb * (KT * 128), &tmK, a.k_col0 + h * DH + kb * 64, tok0 + j * KT, bar_full + 8 * s);
+                    tc::tma_load_2d(sk + kb * (KT * 128), &tmK, a.k_col0 + h * DH + kb * 64, tok0 + j * KT, bar_kfull + 8 * s);
+                issued_k = j + 1;
+                if (!tc::mbar_wait(bar_vempty + 8 * s, ph ^ 1u, &s_abort)) break;
+                const uint32_t sv = tc::smem_u32(sV) + s * V_BYTES;
+                tc::mbar_expect_tx(bar_vfull + 8 * s, V_BYTES);
 #pragma unroll
                 for (int kb = 0; kb < KT / 64; ++kb)
-                    tc::tma_load_2d(sv + kb * (DH * 128), &tmVt, tok0 + j * KT + kb * 64, h * DH, bar_full + 8 * s);
-                issued = j + 1;
+                    tc::tma_load_2d(sv + kb * (DH * 128), &tmVt, tok0 + j * KT + kb * 64, h * DH, bar_vfull + 8 * s);
+                issued_v = j + 1;
             }
             if (s_abort) {
-                for (int j = max(0, issued - KV_STAGES); j < issued; ++j) {
-                    const uint32_t bar = bar_full + 8 * (j % KV_STAGES), ph = (uint32_t)(j / KV_STAGES) & 1u;
+                // give copies already in flight a bounded chance to land before the CTA retires
+                for (int j = max(0, issued_k - KV_STAGES); j < issued_k; ++j) {
+                    const uint32_t bar = bar_kfull + 8 * (j % KV_STAGES), ph = (uint32_t)(j / KV_STAGES) & 1u;
+                    for (int i = 0; i < (1 << 16) && !tc::mbar_try(bar, ph); ++i) {}
+                }
+                for (int j = max(0, issued_v - KV_STAGES); j < issued_v; ++j) {
+                    const uint32_t bar = bar_vfull + 8 * (j % KV_STAGES), ph = (uint32_t)(j / KV_STAGES) & 1u;
                     for (int i = 0; i < (1 << 16) && !tc::mbar_try(bar, ph); ++i) {}
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
-            constexpr uint32_t idesc_s = tc::idesc_bf16_f32(QT, KT);
-            constexpr uint32_t idesc_o = tc::idesc_bf16_f32(QT, DH);
-            auto issue_S = [&](int s) {
-                const uint32_t sk = tc::smem_u32(sKV) + s * STAGE_BYTES;
+        // ---------------- MMA issuer: the whole warp runs the loop with warp-uniform operands, one elected lane issues.
+        // S_{j+1} = Q K_{j+1}^T is issued (into the other S buffer) before O += P_j V_j, so the tensor core computes the next
+        // scores while the softmax warps work on the current ones.
+        constexpr uint32_t idesc_s = tc::idesc_bf16_f32(QT, KT);
+        constexpr uint32_t idesc_o = tc::idesc_bf16_f32(QT, DH);
+        auto issue_S = [&](int j) {
+            const int s = j % KV_STAGES;
+            const uint32_t sk = tc::smem_u32(sK) + s * K_BYTES, d = tmem_S + (uint32_t)(j & 1) * KT;
 #pragma unroll
-                for (int kb = 0; kb < KB; ++kb) {
-                    const uint64_t dq = tc::smem_desc_sw128(tc::smem_u32(sQ) + kb * (QT * 128));
-                    const uint64_t dk = tc::smem_desc_sw128(sk + kb * (KT * 128));
+            for (int kb = 0; kb < KB; ++kb) {
+                const uint64_t dq = tc::smem_desc_sw128(tc::smem_u32(sQ) + kb * (QT * 128));
+                const uint64_t dk = tc::smem_desc_sw128(sk + kb * (KT * 128));
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        tc::mma_bf16(tmem_S, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, (kb | kk) != 0 ? 1u : 0u);
-                }
-                tc::mma_commit(bar_s);
-            };
-            bool ok = tc::mbar_wait(bar_q, 0, &s_abort);
-            for (int j = 0; j < nkv && ok; ++j) {
-                const int s = j % KV_STAGES;
-                if (j == 0) {
-                    ok = tc::mbar_wait(bar_full + 8 * s, 0, &s_abort);
-                    if (!ok) break;
-                    tc::tc_fence_after();
-                    issue_S(s);
-                }
-                ok = tc::mbar_wait(bar_p, (uint32_t)j & 1u, &s_abort);       // P_j is in shared memory, S_j has been read
+                for (int kk = 0; kk < 4; ++kk)
+                    tc::mma_bf16_elect(d, dq + (uint64_t)(kk * 2), dk + (uint64_t)(kk * 2), idesc_s, (kb | kk) != 0 ? 1u : 0u);
+            }
+            tc::mma_commit_elect(bar_s + 8 * (j & 1));
+            tc::mma_commit_elect(bar_kempty + 8 * s);
+        };
+        bool ok = __all_sync(0xffffffffu, tc::mbar_wait(bar_q, 0, &s_abort));
+        ok = ok && __all_sync(0xffffffffu, tc::mbar_wait(bar_kfull, 0, &s_abort));
+        if (ok) { tc::tc_fence_after(); issue_S(0); }
+        for (int j = 0; j < nkv && ok; ++j) {
+            const int s = j % KV_STAGES;
+            if (j + 1 < nkv) {
+                // the S buffer of tile j+1 was last read for tile j-1, before the softmax warps arrived on bar_p (waited below)
+                ok = __all_sync(0xffffffffu, tc::mbar_wait(bar_kfull + 8 * ((j + 1) % KV_STAGES), (uint32_t)((j + 1) / KV_STAGES) & 1u, &s_abort));
                 if (!ok) break;
                 tc::tc_fence_after();
-                const uint32_t sv = tc::smem_u32(sKV) + s * STAGE_BYTES + K_BYTES;
-#pragma unroll
-                for (int kb = 0; kb < KT / 64; ++kb) {
-                    const uint64_t dp = tc::smem_desc_sw128(tc::smem_u32(sP) + kb * (QT * 128));
-                    const uint64_t dv = tc::smem_desc_sw128(sv + kb * (DH * 128));
-#pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)
-                        tc::mma_bf16(tmem_O, dp + (uint64_t)(kk * 2), dv + (uint64_t)(kk * 2), idesc_o, (kb | kk) != 0 ? 1u : 0u);
-                }
-                tc::mma_commit(bar_o);
-                tc::mma_commit(bar_empty + 8 * s);
-                if (j + 1 < nkv) {
-                    const int s1 = (j + 1) % KV_STAGES;
-                    ok = tc::mbar_wait(bar_full + 8 * s1, (uint32_t)((j + 1) / KV_STAGES) & 1u, &s_abort);
-                    if (!ok) break;
-                    tc::tc_fence_after();
-                    issue_S(s1);
-                }
+                issue_S(j + 1);
             }
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(bar_vfull + 8 * s, (uint32_t)(j / KV_STAGES) & 1u, &s_abort));
+            ok = ok && __all_sync(0xffffffffu, tc::mbar_wait(bar_p, (uint32_t)j & 1u, &s_abort));   // P_j written, O rescaled
+            if (!ok) break;
+            tc::tc_fence_after();
+            const uint32_t sv = tc::smem_u32(sV) + s * V_BYTES;
+#pragma unroll
+            for (int kb = 0; kb < KT / 64; ++kb) {
+                const uint64_t dp = tc::smem_desc_sw128(tc::smem_u32(sP) + kb * (QT * 128));
+                const uint64_t dv = tc::smem_desc_sw128(sv + kb * (DH * 128));
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    tc::mma_bf16_elect(tmem_O, dp + (uint64_t)(kk * 2), dv + (uint64_t)(kk * 2), idesc_o, (j | kb | kk) != 0 ? 1u : 0u);
+            }
+            tc::mma_commit_elect(bar_o);
+            tc::mma_commit_elect(bar_vempty + 8 * s);
         }
     } else {
-        // ---------------- online softmax + output accumulation: two threads per query row
+        // ---------------- online softmax: two threads per query row.  O accumulates in tensor memory over the tiles; the
+        // exponentials are taken against a reference maximum that follows the true running maximum lazily: it is moved (and
+        // O and the denominator rescaled) only when the true one has risen by more than 2^8, so most tiles need no pass over O.
         constexpr int HK = KT / 2;                         // keys of a tile per thread
         constexpr int HD = DH / 2;                         // output columns per thread
+        constexpr float kLazy = 8.0f;                      // in log2 units: probabilities stay below 2^8
         const int qd = warp & 3, half = (warp - 2) >> 2;
         const int row = qd * 32 + lane;
         const uint32_t lane_off = (uint32_t)(qd * 32) << 16;
         const float c = a.scale_log2;                      // log2(e) / sqrt(dh)
-        float m = -INFINITY, l = 0.f;                      // l: this thread's keys only; the halves are added at the end
-        float acc[HD];
-#pragma unroll
-        for (int i = 0; i < HD; ++i) acc[i] = 0.f;
+        float m = -INFINITY, l = 0.f;                      // m: reference maximum; l: this thread's keys only
         bool ok = true;
         for (int j = 0; j < nkv && ok; ++j) {
-            ok = tc::mbar_wait(bar_s, (uint32_t)j & 1u, &s_abort);
+            ok = tc::mbar_wait(bar_s + 8 * (j & 1), (uint32_t)(j >> 1) & 1u, &s_abort);
             if (!ok) break;
             tc::tc_fence_after();
             const int valid = min(KT, S - j * KT) - half * HK;     // keys of this thread's half that belong to the sequence
             uint32_t v[HK];
 #pragma unroll
-            for (int cc = 0; cc < HK / 32; ++cc) tc::tmem_ld32(tmem_S + lane_off + half * HK + cc * 32, v + cc * 32);
+            for (int cc = 0; cc < HK / 32; ++cc) tc::tmem_ld32(tmem_S + (uint32_t)(j & 1) * KT + lane_off + half * HK + cc * 32, v + cc * 32);
             tc::tmem_ld_wait();
+            const bool full = valid >= HK;                 // uniform over the warp: no per-key test on whole tiles
             float mx = -INFINITY;
+            if (full) {
+                float mx1 = -INFINITY;
 #pragma unroll
-            for (int i = 0; i < HK; ++i)
-                if (i < valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+                for (int i = 0; i < HK; i += 2) { mx = fmaxf(mx, __uint_as_float(v[i])); mx1 = fmaxf(mx1, __uint_as_float(v[i + 1])); }
+                mx = fmaxf(mx, mx1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < HK; ++i)
+                    if (i < valid) mx = fmaxf(mx, __uint_as_float(v[i]));
+            }
             s_xch[j & 1][half][row] = mx;                  // exchange the two halves' maxima (bounded wait, like every other)
             tc::mbar_arrive(bar_x);
             ok = tc::mbar_wait(bar_x, (uint32_t)j & 1u, &s_abort);
             if (!ok) break;
-            const float m_new = fmaxf(m, fmaxf(mx, s_xch[j & 1][half ^ 1][row]));
-            const float alpha = exp2f((m - m_new) * c);
-            const float mc = m_new * c;
-            float lsum = 0.f;
+            const float m_row = fmaxf(mx, s_xch[j & 1][half ^ 1][row]);   // both threads of a row see the same value
+            if (j == 0) {
+                m = m_row;
+            } else {
+                // P_{j-1} V_{j-1} has finished: O may be rescaled, and the P buffer rewritten
+                ok = tc::mbar_wait(bar_o, (uint32_t)(j - 1) & 1u, &s_abort);
+                if (!ok) break;
+                const bool move = (m_row - m) * c > kLazy;
+                if (__any_sync(0xffffffffu, move)) {
+                    tc::tc_fence_after();
+                    const float alpha = move ? tc::ex2_approx((m - m_row) * c) : 1.0f;
+#pragma unroll
+                    for (int cc = 0; cc < HD / 32; ++cc) {
+                        uint32_t o[32];
+                        tc::tmem_ld32(tmem_O + lane_off + half * HD + cc * 32, o);
+                        tc::tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tc::tmem_st32(tmem_O + lane_off + half * HD + cc * 32, o);
+                    }
+                    tc::tmem_st_wait();
+                    if (move) { l *= alpha; m = m_row; }
+                }
+            }
+            const float mc = m * c;
+            float lsum = 0.f, lsum1 = 0.f;
 #pragma unroll
             for (int cc = 0; cc < HK / 32; ++cc) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float p0 = (cc * 32 + 2 * i < valid) ? exp2f(fmaf(__uint_as_float(v[cc * 32 + 2 * i]), c, -mc)) : 0.f;
-                    const float p1 = (cc * 32 + 2 * i + 1 < valid) ? exp2f(fmaf(__uint_as_float(v[cc * 32 + 2 * i + 1]), c, -mc)) : 0.f;
-                    lsum += p0 + p1;
+                    float p0 = tc::ex2_approx(fmaf(__uint_as_float(v[cc * 32 + 2 * i]), c, -mc));
+                    float p1 = tc::ex2_approx(fmaf(__uint_as_float(v[cc * 32 + 2 * i + 1]), c, -mc));
+                    if (!full) {
+                        if (cc * 32 + 2 * i >= valid) p0 = 0.f;
+                        if (cc * 32 + 2 * i + 1 >= valid) p1 = 0.f;
+                    }
+                    if (i & 1) lsum1 += p0 + p1; else lsum += p0 + p1;
                     __nv_bfloat162 hh = __floats2bfloat162_rn(p0, p1);
                     pk[i] = *reinterpret_cast<uint32_t *>(&hh);
                 }
@@ -197,40 +247,38 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
                     *reinterpret_cast<uint4 *>(prow + chunk * 16) = make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
                 }
             }
-            l = l * alpha + lsum;
-            m = m_new;
+            l += lsum + lsum1;
             tc::fence_proxy_async_smem();                  // P visible to the tensor core's shared-memory reads
-            tc::tc_fence_before();
+            tc::tc_fence_before();                         // S_j has been read, O has been rescaled
             tc::mbar_arrive(bar_p);
-            ok = tc::mbar_wait(bar_o, (uint32_t)j & 1u, &s_abort);
-            if (!ok) break;
-            tc::tc_fence_after();
-#pragma unroll
-            for (int cc = 0; cc < HD / 32; ++cc) {
-                uint32_t o[32];
-                tc::tmem_ld32(tmem_O + lane_off + half * HD + cc * 32, o);
-                tc::tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) acc[cc * 32 + i] = fmaf(acc[cc * 32 + i], alpha, __uint_as_float(o[i]));
-            }
-            tc::tc_fence_before();
         }
-        // the two halves of a row add their partial denominators
+        // the last P V, then the two halves of a row add their partial denominators
+        ok = ok && tc::mbar_wait(bar_o, (uint32_t)(nkv - 1) & 1u, &s_abort);
         s_xch[nkv & 1][half][row] = l;
         tc::mbar_arrive(bar_x);
         ok = ok && tc::mbar_wait(bar_x, (uint32_t)nkv & 1u, &s_abort);
-        if (ok && !s_abort && q0 + row < a.kq) {
+        if (ok && !s_abort) {
+            tc::tc_fence_after();
             const float inv = 1.0f / (l + s_xch[nkv & 1][half ^ 1][row]);
+            const bool live = q0 + row < a.kq;
             __nv_bfloat16 *dst = a.out + (long long)(qrow0 + row) * a.ld_out + h * DH + half * HD;
 #pragma unroll
-            for (int i = 0; i < HD / 8; ++i) {
-                uint32_t o[4];
+            for (int cc = 0; cc < HD / 32; ++cc) {
+                uint32_t o[32];
+                tc::tmem_ld32(tmem_O + lane_off + half * HD + cc * 32, o);      // warp-collective: every lane takes part
+                tc::tmem_ld_wait();
+                if (live) {
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    __nv_bfloat162 hh = __floats2bfloat162_rn(acc[8 * i + 2 * t] * inv, acc[8 * i + 2 * t + 1] * inv);
-                    o[t] = *reinterpret_cast<uint32_t *>(&hh);
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            __nv_bfloat162 hh = __floats2bfloat162_rn(__uint_as_float(o[8 * i + 2 * t]) * inv, __uint_as_float(o[8 * i + 2 * t + 1]) * inv);
+                            w[t] = *reinterpret_cast<uint32_t *>(&hh);
+                        }
+                        reinterpret_cast<uint4 *>(dst)[cc * 4 + i] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
                 }
-                reinterpret_cast<uint4 *>(dst)[i] = make_uint4(o[0], o[1], o[2], o[3]);
             }
         }
     }
@@ -245,7 +293,7 @@ template <int DH>
 int32_t launch_dh(const AttnPlan &p, int kq, const int32_t *d_active, int32_t *err, cudaStream_t stream)
 {
     constexpr size_t smem = (size_t)QT * DH * 2 + KV_STAGES * (size_t)(KT * DH * 2 + DH * KT * 2) + QT * KT * 2
-                          + (2 * KV_STAGES + 5) * 8 + 16 + 1024;
+                          + kAttnBars * 8 + 16 + 1024;
     static bool configured = false;
     if (!configured) {
         SFS_CUDA(cudaFuncSetAttribute(attention_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -418,6 +418,7 @@ int stages_for(int mb, int bn)
 // (MB*128 + bn/2) rows x 128 B at the ~40 B/clk an SM sustains from L2 when every SM streams; below ~750 clocks the
 // k-block time stops shrinking with the tile (load latency over the bytes a CTA can keep in flight).  All measured.
 // The epilogue hides behind the next tile when two accumulators fit tensor memory, except for a pair's last tile.
+// Splitting K pays for few rows only: the slabs grow with M, the idle pairs they avoid do not.
 long long model_clocks(int M, int K, int mode, int n_maps, int n_per_map, int pairs, int mb, int bn, int splits)
 {
     const long long num_kb = (K + BK - 1) / BK, kbps = (num_kb + splits - 1) / splits;
@@ -429,7 +430,10 @@ long long model_clocks(int M, int K, int mode, int n_maps, int n_per_map, int pa
     if (kb_clk < 750) kb_clk = 750;
     const long long epi = (long long)mb * bn * 16 + 3000;
     const bool hidden = mb * ((bn + 31) & ~31) <= 256;
-    return waves * kbps * kb_clk + (hidden ? 1 : waves) * epi + (splits > 1 ? 1500LL * splits : 0);
+    // a split K also costs the fp32 slab that the next RMSNorm reads back: M x N x 4 bytes, measured at ~1.2e-3 clocks per element
+    const long long n_out = (mode == GEMM_SWIGLU) ? n_per_map : (long long)n_maps * n_per_map;
+    const long long slab = 1500 + (long long)((double)M * (double)n_out * 1.2e-3);
+    return waves * kbps * kb_clk + (hidden ? 1 : waves) * epi + (splits > 1 ? slab * splits : 0);
 }
 
 // Tile shape (MB blocks of 256 rows, width bn) and number of K ranges with the smallest modelled time.  Wide, tall tiles
