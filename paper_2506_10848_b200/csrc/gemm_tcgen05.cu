@@ -67,7 +67,8 @@ constexpr int kBarBytes = (2 * kMaxStages + 4) * 8 + 16;
 constexpr int kTmemCols = 512;
 constexpr int kEpiStageBytes = kEpiWarps * 32 * 128;   // one 32-row x 128-byte output unit per epilogue warp
 
-__device__ __forceinline__ float silu_f(float x) { return x / (1.0f + __expf(-x)); }
+// x * sigmoid(x) with the special-function unit's exponential and reciprocal (a few ulp: the result is rounded to bf16)
+__device__ __forceinline__ float silu_f(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -157,78 +158,102 @@ __device__ __forceinline__ void flush_unit(const GemmArgs &g, long long slab, ui
 
 // One warp's share of a tile's epilogue: TMEM lane quarter q (32 rows) of every 256-row block, the units of parity `par`.
 // A unit may reach past the tile's valid columns: those accumulator columns exist (inside the 256-column buffer) and
-// are never stored.
+// are never stored.  The tensor-memory loads of the next piece are issued as soon as the current piece has been
+// converted, so their latency hides behind the parking and the stores of the current one.
 __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord &t, uint32_t tmem_acc, uint32_t bn_pad, uint32_t stage,
                                               int q, int par, int lane, int rank, int M)
 {
     const int HALF = g.bn >> 1;
     const int lim = min(t.ncol0 + t.ncols, g.N);         // first output column this tile must not touch
-    for (int b = 0; b < g.mb; ++b) {
-        const int grow0 = t.m0 + b * 2 * BM + rank * BM + q * 32;
-        const uint32_t tbase = tmem_acc + b * bn_pad + ((uint32_t)(q * 32) << 16);
-        if (g.mode == GEMM_SWIGLU) {
-            for (int c = 64 * par; c < t.ncols; c += 128) {             // 64 outputs = 64 gate + 64 up columns
+    const uint32_t tq = tmem_acc + ((uint32_t)(q * 32) << 16);
+    const int grow_q = t.m0 + rank * BM + q * 32;        // first row of block 0 handled by this warp
+    if (g.mode == GEMM_SWIGLU || (g.mode == GEMM_STORE && !g.out_f32 && !(g.vt != nullptr && t.ncol0 >= g.vt_col0))) {
+        // ---- bf16 output (plain or SwiGLU): units of 64 output columns, handled as two pieces of 32
+        const bool swiglu = (g.mode == GEMM_SWIGLU);
+        const int upb = (t.ncols - 64 * par + 127) / 128;                 // units per 256-row block for this parity (>= 0)
+        const int n_pieces = upb > 0 ? 2 * upb * g.mb : 0;
+        auto piece_addr = [&](int pc) {                                   // tensor-memory column of piece pc
+            const int u = pc >> 1, b = u / upb, c = 64 * par + 128 * (u - b * upb);
+            return tq + (uint32_t)(b * bn_pad + c + 32 * (pc & 1));
+        };
+        uint32_t x0[32], x1[32];
+        if (n_pieces > 0) {
+            tc::tmem_ld32(piece_addr(0), x0);
+            if (swiglu) tc::tmem_ld32(piece_addr(0) + HALF, x1);
+        }
+        for (int pc = 0; pc < n_pieces; ++pc) {
+            uint32_t o[16];
+            tc::tmem_ld_wait32(x0);
+            if (swiglu) tc::tmem_ld_wait32(x1);
+            if (swiglu) {
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t gt[32], up[32], o[16];
-                    tc::tmem_ld32(tbase + c + 32 * h, gt);
-                    tc::tmem_ld32(tbase + HALF + c + 32 * h, up);
-                    tc::tmem_ld_wait();
+                for (int j = 0; j < 16; ++j)
+                    o[j] = pack_bf16(silu_f(__uint_as_float(x0[2 * j])) * __uint_as_float(x1[2 * j]),
+                                     silu_f(__uint_as_float(x0[2 * j + 1])) * __uint_as_float(x1[2 * j + 1]));
+            } else {
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        o[j] = pack_bf16(silu_f(__uint_as_float(gt[2 * j])) * __uint_as_float(up[2 * j]),
-                                         silu_f(__uint_as_float(gt[2 * j + 1])) * __uint_as_float(up[2 * j + 1]));
-                    park16(stage, lane, 4 * h, o);
-                }
+                for (int j = 0; j < 16; ++j) o[j] = pack_bf16(__uint_as_float(x0[2 * j]) * g.scale, __uint_as_float(x0[2 * j + 1]) * g.scale);
+            }
+            if (pc + 1 < n_pieces) {
+                tc::tmem_ld32(piece_addr(pc + 1), x0);
+                if (swiglu) tc::tmem_ld32(piece_addr(pc + 1) + HALF, x1);
+            }
+            park16(stage, lane, 4 * (pc & 1), o);
+            if (pc & 1) {
+                const int u = pc >> 1, b = u / upb, c = 64 * par + 128 * (u - b * upb);
                 __syncwarp();
-                flush_unit<2, false>(g, 0, stage, lane, grow0, M, t.ncol0 + c, lim);
+                flush_unit<2, false>(g, 0, stage, lane, grow_q + b * 2 * BM, M, t.ncol0 + c, lim);
                 __syncwarp();
             }
-        } else if (g.vt != nullptr && t.ncol0 >= g.vt_col0) {
-            // V columns of the QKV projection go out transposed: the 32 lanes hold 32 consecutive tokens of a feature
-            const int grow = grow0 + lane;
-            for (int c = 32 * par; c < t.ncols; c += 64) {
-                uint32_t v[32];
-                tc::tmem_ld32(tbase + c, v);
-                tc::tmem_ld_wait();
-                if (grow < M) {
+        }
+    } else if (g.vt != nullptr && t.ncol0 >= g.vt_col0) {
+        // ---- V columns of the QKV projection go out transposed: the 32 lanes hold 32 consecutive tokens of a feature
+        const int upb = (t.ncols - 32 * par + 63) / 64;
+        const int n_pieces = upb > 0 ? upb * g.mb : 0;
+        auto piece_col = [&](int pc, int *b) { *b = pc / upb; return 32 * par + 64 * (pc - *b * upb); };
+        uint32_t v[32];
+        int b0;
+        if (n_pieces > 0) { const int c = piece_col(0, &b0); tc::tmem_ld32(tq + (uint32_t)(b0 * bn_pad + c), v); }
+        for (int pc = 0; pc < n_pieces; ++pc) {
+            int b;
+            const int c = piece_col(pc, &b);
+            uint16_t h[32];
+            tc::tmem_ld_wait32(v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (t.ncol0 + c + j < lim)
-                            g.vt[(long long)(t.ncol0 + c + j - g.vt_col0) * g.ldvt + grow] = __float2bfloat16_rn(__uint_as_float(v[j]) * g.scale);
-                }
+            for (int j = 0; j < 32; ++j) { __nv_bfloat16 r = __float2bfloat16_rn(__uint_as_float(v[j]) * g.scale); h[j] = *reinterpret_cast<uint16_t *>(&r); }
+            if (pc + 1 < n_pieces) { int bn2; const int c2 = piece_col(pc + 1, &bn2); tc::tmem_ld32(tq + (uint32_t)(bn2 * bn_pad + c2), v); }
+            const int grow = grow_q + b * 2 * BM + lane;
+            if (grow < M) {
+                uint16_t *dst = reinterpret_cast<uint16_t *>(g.vt) + (long long)(t.ncol0 + c - g.vt_col0) * g.ldvt + grow;
+                const int nv = lim - (t.ncol0 + c);                        // valid features of this piece
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (j < nv) dst[(long long)j * g.ldvt] = h[j];
             }
-        } else if (g.mode == GEMM_RESIDUAL_F32 || g.out_f32) {
-            for (int c = 32 * par; c < t.ncols; c += 64) {              // 32 fp32 columns
-                uint32_t v[32];
-                tc::tmem_ld32(tbase + c, v);
-                tc::tmem_ld_wait();
-                if (g.mode != GEMM_RESIDUAL_F32 && g.scale != 1.0f) {
+        }
+    } else {
+        // ---- fp32 output (residual add, split-K slab, or fp32 logits): units of 32 columns
+        const int upb = (t.ncols - 32 * par + 63) / 64;
+        const int n_pieces = upb > 0 ? upb * g.mb : 0;
+        auto piece_col = [&](int pc, int *b) { *b = pc / upb; return 32 * par + 64 * (pc - *b * upb); };
+        const bool scale = (g.mode != GEMM_RESIDUAL_F32 && g.scale != 1.0f);
+        uint32_t v[32];
+        int b0;
+        if (n_pieces > 0) { const int c = piece_col(0, &b0); tc::tmem_ld32(tq + (uint32_t)(b0 * bn_pad + c), v); }
+        for (int pc = 0; pc < n_pieces; ++pc) {
+            int b;
+            const int c = piece_col(pc, &b);
+            uint32_t o[32];
+            tc::tmem_ld_wait32(v);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * g.scale);
-                }
-                park16(stage, lane, 0, v);
-                park16(stage, lane, 4, v + 16);
-                __syncwarp();
-                if (g.mode == GEMM_RESIDUAL_F32 && g.splits == 1) flush_unit<4, true>(g, 0, stage, lane, grow0, M, t.ncol0 + c, lim);
-                else flush_unit<4, false>(g, (long long)t.split * g.split_stride, stage, lane, grow0, M, t.ncol0 + c, lim);
-                __syncwarp();
-            }
-        } else {
-            for (int c = 64 * par; c < t.ncols; c += 128) {             // 64 bf16 columns
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t v[32], o[16];
-                    tc::tmem_ld32(tbase + c + 32 * h, v);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 16; ++j) o[j] = pack_bf16(__uint_as_float(v[2 * j]) * g.scale, __uint_as_float(v[2 * j + 1]) * g.scale);
-                    park16(stage, lane, 4 * h, o);
-                }
-                __syncwarp();
-                flush_unit<2, false>(g, 0, stage, lane, grow0, M, t.ncol0 + c, lim);
-                __syncwarp();
-            }
+            for (int j = 0; j < 32; ++j) o[j] = scale ? __float_as_uint(__uint_as_float(v[j]) * g.scale) : v[j];
+            if (pc + 1 < n_pieces) { int bn2; const int c2 = piece_col(pc + 1, &bn2); tc::tmem_ld32(tq + (uint32_t)(bn2 * bn_pad + c2), v); }
+            park16(stage, lane, 0, o);
+            park16(stage, lane, 4, o + 16);
+            __syncwarp();
+            if (g.mode == GEMM_RESIDUAL_F32 && g.splits == 1) flush_unit<4, true>(g, 0, stage, lane, grow_q + b * 2 * BM, M, t.ncol0 + c, lim);
+            else flush_unit<4, false>(g, (long long)t.split * g.split_stride, stage, lane, grow_q + b * 2 * BM, M, t.ncol0 + c, lim);
+            __syncwarp();
         }
     }
 }
