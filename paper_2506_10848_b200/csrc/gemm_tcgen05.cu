@@ -170,10 +170,11 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
     if (g.mode == GEMM_SWIGLU || (g.mode == GEMM_STORE && !g.out_f32 && !(g.vt != nullptr && t.ncol0 >= g.vt_col0))) {
         // ---- bf16 output (plain or SwiGLU): units of 64 output columns, handled as two pieces of 32
         const bool swiglu = (g.mode == GEMM_SWIGLU);
-        const int upb = (t.ncols - 64 * par + 127) / 128;                 // units per 256-row block for this parity (>= 0)
-        const int n_pieces = upb > 0 ? 2 * upb * g.mb : 0;
+        // the units of all 256-row blocks, numbered block by block, alternate between the two warps of a lane quarter
+        const int upb = (t.ncols + 63) / 64;                              // units per 256-row block
+        const int n_pieces = 2 * ((g.mb * upb - par + 1) / 2);
         auto piece_addr = [&](int pc) {                                   // tensor-memory column of piece pc
-            const int u = pc >> 1, b = u / upb, c = 64 * par + 128 * (u - b * upb);
+            const int u = par + 2 * (pc >> 1), b = u / upb, c = 64 * (u - b * upb);
             return tq + (uint32_t)(b * bn_pad + c + 32 * (pc & 1));
         };
         uint32_t x0[32], x1[32];
@@ -200,7 +201,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
             }
             park16(stage, lane, 4 * (pc & 1), o);
             if (pc & 1) {
-                const int u = pc >> 1, b = u / upb, c = 64 * par + 128 * (u - b * upb);
+                const int u = par + 2 * (pc >> 1), b = u / upb, c = 64 * (u - b * upb);
                 __syncwarp();
                 flush_unit<2, false>(g, 0, stage, lane, grow_q + b * 2 * BM, M, t.ncol0 + c, lim);
                 __syncwarp();
@@ -208,9 +209,9 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
         }
     } else if (g.vt != nullptr && t.ncol0 >= g.vt_col0) {
         // ---- V columns of the QKV projection go out transposed: the 32 lanes hold 32 consecutive tokens of a feature
-        const int upb = (t.ncols - 32 * par + 63) / 64;
-        const int n_pieces = upb > 0 ? upb * g.mb : 0;
-        auto piece_col = [&](int pc, int *b) { *b = pc / upb; return 32 * par + 64 * (pc - *b * upb); };
+        const int upb = (t.ncols + 31) / 32;
+        const int n_pieces = (g.mb * upb - par + 1) / 2;
+        auto piece_col = [&](int pc, int *b) { const int u = par + 2 * pc; *b = u / upb; return 32 * (u - *b * upb); };
         uint32_t v[32];
         int b0;
         if (n_pieces > 0) { const int c = piece_col(0, &b0); tc::tmem_ld32(tq + (uint32_t)(b0 * bn_pad + c), v); }
@@ -233,9 +234,9 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
         }
     } else {
         // ---- fp32 output (residual add, split-K slab, or fp32 logits): units of 32 columns
-        const int upb = (t.ncols - 32 * par + 63) / 64;
-        const int n_pieces = upb > 0 ? upb * g.mb : 0;
-        auto piece_col = [&](int pc, int *b) { *b = pc / upb; return 32 * par + 64 * (pc - *b * upb); };
+        const int upb = (t.ncols + 31) / 32;
+        const int n_pieces = (g.mb * upb - par + 1) / 2;
+        auto piece_col = [&](int pc, int *b) { const int u = par + 2 * pc; *b = u / upb; return 32 * (u - *b * upb); };
         const bool scale = (g.mode != GEMM_RESIDUAL_F32 && g.scale != 1.0f);
         uint32_t v[32];
         int b0;
