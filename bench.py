@@ -442,8 +442,8 @@ def main():
     roofline = {"bound": "tensor", "achieved": res["gemm_tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": (res["gemm_tflops"] / peaks["bf16_tflops_sustained"]) if res["gemm_tflops"] else None,
                 # DRAM read + write bytes per GEMM launch from one ncu capture of this kernel on the 2-layer case, scaled to
-                # the 129 launches of a full step (32 x 484.0 MB + 1.05 GB LM head); the shape of the main workload only
-                "traffic": (16.54e9 / 129.0) if (args.workload == "8b" and not args.layers) else None,
+                # the 129 launches of a full step (32 x 484.8 MB + 1.05 GB LM head); the shape of the main workload only
+                "traffic": (16.57e9 / 129.0) if (args.workload == "8b" and not args.layers) else None,
                 "kernel": "gemm_kernel (tcgen05 projections: QKV, O, gate/up+SwiGLU, down, LM head)",
                 "peak_source": peaks["source"] + " (sustained cuBLAS bf16, kernel timed inside a long step)",
                 "launches_timed": res["gemm_launches"], "ms_timed": res["gemm_ms"], "steps_timed": res["prof_steps"]}
