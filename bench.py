@@ -223,9 +223,8 @@ def time_back_to_back(torch, fn, n):
     return e0.elapsed_time(e1) / n
 
 
-def run_extras(torch, sfs, W, model, shape, dev, peaks):
-    """The other workloads of the benchmark definition, measured on the same model: the sampling-epilogue
-    microbenchmark, the cached run (prompt 1024 + 512 masked) and the batch of 8 sequences (512 + 256)."""
+def run_epilogue(torch, sfs, W, shape, dev, peaks):
+    """The sampling-epilogue microbenchmark: row statistics on cold bf16 logits, one slow and one fast selection step."""
     out = {}
     V = shape.vocab
     # ---- sampling epilogue: bf16 [256, V] logits with planted winners; 4 rotating copies (259 MB > L2) keep every launch cold
@@ -261,6 +260,15 @@ def run_extras(torch, sfs, W, model, shape, dev, peaks):
                        "select_fast_step_us": fast_us, "span": [lo, hi]}
     del bufs
     torch.cuda.empty_cache()
+    return out
+
+
+def run_extras(torch, sfs, W, model, shape, dev, peaks):
+    """The other workloads of the benchmark definition, measured on the same model: the sampling-epilogue
+    microbenchmark, the cached run (prompt 1024 + 512 masked) and the batch of 8 sequences (512 + 256)."""
+    out = run_epilogue(torch, sfs, W, shape, dev, peaks)
+    V = shape.vocab
+    params = sfs.Params.default()
 
     def timed_steps(session, n):
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
@@ -406,6 +414,7 @@ def main():
     ap.add_argument("--no-e2e", dest="e2e", action="store_false")
     ap.add_argument("--no-extras", dest="extras", action="store_false", help="skip the epilogue / cached / batch-8 workloads")
     ap.add_argument("--no-cpu-baseline", dest="cpu", action="store_false")
+    ap.add_argument("--epilogue-only", action="store_true", help="run only the sampling-epilogue microbenchmark (small case for ncu captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", 0))
@@ -424,6 +433,14 @@ def main():
         entry.build()
     if world > 1:
         torch.distributed.barrier()
+    if args.epilogue_only:
+        # a profiling case, not a bench line: the microbenchmark alone (260 MB on the device)
+        if rank == 0:
+            from paper_2506_10848_b200 import binding as sfs
+            from paper_2506_10848_b200 import workloads as W
+            torch.cuda.set_device(0)
+            print(json.dumps({"profiling_case": "sampling epilogue only", **run_epilogue(torch, sfs, W, W.LLADA_8B, "cuda:0", measured_peaks())}))
+        return
     res = run_ours(args, rank, world)
 
     ms, tokens = res["ms"], res["tokens"]

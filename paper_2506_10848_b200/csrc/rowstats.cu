@@ -79,6 +79,9 @@ __device__ __forceinline__ uint32_t canon_pair(uint32_t w, const Consts2 &k) {
     return shr_clamp(p0 << 9, kShiftBase - r0) + shr_clamp(p1 << 9, kShiftBase - r1);
 }
 
+// orders this thread's shared-memory traffic inside the cluster (cheaper than a device-wide fence)
+__device__ __forceinline__ void cluster_fence() { asm volatile("fence.acq_rel.cluster;" ::: "memory"); }
+
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
@@ -215,13 +218,13 @@ rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int
             int *ra = cluster.map_shared_rank(&s_row_arg, 0), *rn = cluster.map_shared_rank(&s_arrived, 0);
             atomicAdd(rs, t);
             atomicMin(ra, arg);
-            __threadfence();
+            cluster_fence();
             atomicAdd(rn, 1);
             if (rank == 0) {
                 int spins = 0;
                 while (*reinterpret_cast<volatile int *>(&s_arrived) < C && ++spins < (1 << 24)) {}
                 if (spins >= (1 << 24) && err) atomicExch(err, SFS_ERR_TIMEOUT);   // a peer never reported
-                __threadfence();
+                cluster_fence();
                 const int a2 = *reinterpret_cast<volatile int *>(&s_row_arg);
                 write_row(out, row, a2 == 0x7FFFFFFF ? 0 : a2, *reinterpret_cast<volatile unsigned long long *>(&s_row_sum));
             }
@@ -229,6 +232,151 @@ rowstats_cluster_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int
             write_row(out, row, arg == 0x7FFFFFFF ? 0 : arg, t);
         }
     }
+}
+
+// ---- long rows: slices staged in shared memory ------------------------------------------------------------------
+// Same arithmetic, other staging: a cluster of 8 CTAs of 128 threads owns a row, and each CTA brings its contiguous slice
+// into shared memory with ONE bulk asynchronous copy, so no registers are tied up while the bytes are in flight and seven
+// CTAs (seven 32 KB slices) fit an SM instead of four.  The two passes then read shared memory.
+constexpr int kStagedThreads = 128;
+constexpr int kStagedCluster = 8;
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__global__ void __launch_bounds__(kStagedThreads)
+rowstats_staged_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int nchunks, int per_cta, int vocab,
+                     const int32_t *__restrict__ n_rows_ptr, int max_rows, RowOut out, int32_t *err)
+{
+    cg::cluster_group cluster = cg::this_cluster();
+    const int C    = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    const int row  = blockIdx.x / C;
+    const int n_rows = n_rows_ptr ? min(*n_rows_ptr, max_rows) : max_rows;
+    if (row >= n_rows) return;                              // uniform over the cluster
+
+    extern __shared__ __align__(16) uint4 s_slice[];
+    __shared__ __align__(8) unsigned long long s_bar;
+    __shared__ float s_wmax[kStagedThreads / 32];
+    __shared__ unsigned long long s_wsum[kStagedThreads / 32];
+    __shared__ float s_max_of[kStagedCluster];
+    __shared__ unsigned long long s_row_sum;
+    __shared__ int s_row_arg, s_arrived, s_cta_arg;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int c0 = rank * per_cta;                          // first 16-byte chunk of this CTA's slice
+    const int n = max(0, min(per_cta, nchunks - c0));
+    const uint32_t bar = smem_addr(&s_bar);
+    if (tid == 0) {
+        s_cta_arg = 0x7FFFFFFF; s_row_sum = 0; s_row_arg = 0x7FFFFFFF; s_arrived = 0;
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (n > 0) {
+            const uint32_t bytes = (uint32_t)n * 16u;
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(smem_addr(s_slice)), "l"(logits + (long long)row * ld_chunks + c0), "r"(bytes), "r"(bar) : "memory");
+        } else {
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+        }
+    }
+    __syncthreads();
+    {   // bounded wait for the slice; on expiry the status word is set and the row's result is meaningless
+        uint32_t ok = 0;
+        for (int i = 0; i < (1 << 20) && !ok; ++i)
+            asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                         : "=r"(ok) : "r"(bar) : "memory");
+        if (!ok && err) atomicExch(err, SFS_ERR_TIMEOUT);
+    }
+
+    // ---- pass 1: exact maximum
+    __nv_bfloat162 mx = as_bf162(kNegInf2);
+    for (int c = tid; c < n; c += kStagedThreads) {
+        const uint4 v = s_slice[c];
+        mx = __hmax2(mx, __hmax2(__hmax2(as_bf162(v.x), as_bf162(v.y)), __hmax2(as_bf162(v.z), as_bf162(v.w))));
+    }
+    const float lmax = bf162_max(*reinterpret_cast<uint32_t *>(&mx));
+    float m = warp_max(lmax);
+    if (lane == 0) s_wmax[warp] = m;
+    __syncthreads();
+    if (tid < C) {
+        float t = s_wmax[0];
+#pragma unroll
+        for (int w = 1; w < kStagedThreads / 32; ++w) t = fmaxf(t, s_wmax[w]);
+        *cluster.map_shared_rank(&s_max_of[rank], tid) = t;
+    }
+    cluster.sync();                                         // the only cluster barrier: all slice maxima are here
+    m = s_max_of[0];
+    for (int r = 1; r < C; ++r) m = fmaxf(m, s_max_of[r]);
+
+    // ---- first position of the maximum (only threads that hold it look), then pass 2
+    if (lmax == m) {
+        int best = 0x7FFFFFFF;
+        for (int c = tid; c < n && best == 0x7FFFFFFF; c += kStagedThreads) {
+            const uint4 v = s_slice[c];
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int e = 7; e >= 0; --e) {
+                const float x = (e & 1) ? __uint_as_float(w[e >> 1] & 0xFFFF0000u) : __uint_as_float(w[e >> 1] << 16);
+                const int idx = (c0 + c) * 8 + e;
+                if (x == m && idx < vocab) best = idx;
+            }
+        }
+        if (best != 0x7FFFFFFF) atomicMin(&s_cta_arg, best);
+    }
+    Consts2 k;
+    k.negm = pack2(-m, -m);           k.l2e = pack2(kLog2e, kLog2e);
+    k.magic = pack2(kMagic, kMagic);  k.negmagic = pack2(-kMagic, -kMagic);
+    k.negln2 = pack2(-kLn2, -kLn2);
+    k.c1 = pack2(kC1, kC1); k.c2 = pack2(kC2, kC2); k.c3 = pack2(kC3, kC3); k.c4 = pack2(kC4, kC4);
+    k.three = pack2(3.0f, 3.0f);
+    unsigned long long acc = 0;
+#pragma unroll 4
+    for (int c = tid; c < n; c += kStagedThreads) {
+        const uint4 v = s_slice[c];
+        const uint32_t a = canon_pair(v.x, k) + canon_pair(v.y, k) + canon_pair(v.z, k) + canon_pair(v.w, k);
+        acc += a;                                           // 8 terms < 8 * 1.42 * 2^28 < 2^32
+    }
+    acc = warp_sum_u64(acc);
+    if (lane == 0) s_wsum[warp] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned long long t = 0;
+#pragma unroll
+        for (int w = 0; w < kStagedThreads / 32; ++w) t += s_wsum[w];
+        const int arg = s_cta_arg;
+        unsigned long long *rs = cluster.map_shared_rank(&s_row_sum, 0);
+        int *ra = cluster.map_shared_rank(&s_row_arg, 0), *rn = cluster.map_shared_rank(&s_arrived, 0);
+        atomicAdd(rs, t);
+        atomicMin(ra, arg);
+        cluster_fence();
+        atomicAdd(rn, 1);
+        if (rank == 0) {
+            int spins = 0;
+            while (*reinterpret_cast<volatile int *>(&s_arrived) < C && ++spins < (1 << 24)) {}
+            if (spins >= (1 << 24) && err) atomicExch(err, SFS_ERR_TIMEOUT);   // a peer never reported
+            cluster_fence();
+            const int a2 = *reinterpret_cast<volatile int *>(&s_row_arg);
+            write_row(out, row, a2 == 0x7FFFFFFF ? 0 : a2, *reinterpret_cast<volatile unsigned long long *>(&s_row_sum));
+        }
+    }
+}
+
+int32_t launch_staged(const uint4 *logits, long long ld_chunks, int nchunks, int vocab, const int32_t *d_n_rows,
+                      int max_rows, const RowOut &out, cudaStream_t stream)
+{
+    const int per_cta = (nchunks + kStagedCluster - 1) / kStagedCluster;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(max_rows * kStagedCluster), 1, 1);
+    cfg.blockDim = dim3(kStagedThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)per_cta * 16;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)kStagedCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_staged_bf16, logits, ld_chunks, nchunks, per_cta, vocab, d_n_rows, max_rows, out,
+                                device_status_word_if_any()));
+    return SFS_OK;
 }
 
 // ---- generic path ------------------------------------------------------------------------------------
@@ -314,6 +462,9 @@ int32_t launch_row_stats(const void *d_logits, int32_t logits_dtype, int32_t voc
     const bool fast = logits_dtype == SFS_LOGITS_BF16 && (vocab % 8) == 0 && (ld % 8) == 0 && aligned_to(d_logits, 16);
     if (fast) {
         const int nchunks = vocab / 8;
+        // long rows (128 KB and more, slices of at most 40 KB): staged through shared memory
+        if (nchunks >= 8192 && (nchunks + kStagedCluster - 1) / kStagedCluster <= 2560)
+            return launch_staged(reinterpret_cast<const uint4 *>(d_logits), ld / 8, nchunks, vocab, d_n_rows, max_rows, out, stream);
         // smallest (cluster size, chunks per thread) that covers the row; at most 8 CTAs x 256 threads x 8 chunks
         const int per_cta1 = kThreads;                      // chunks covered by one CTA with NV = 1
         int C = 1, NV = 1;
