@@ -208,7 +208,9 @@ int32_t sfs_cache_reset(sfs_session *session);
 /* One cached forward step (as sfs_forward, for B sequences of P prompt + (S - P) response tokens); advances the step
  * counter.  d_state [B] (optional) tells slow from fast steps and gives the span; NULL means slow.  Optional dumps:
  * d_sets int32 [n_layers, B, n_sel] receives the recomputed token indices of every layer (n_sel as returned in *n_sel,
- * a HOST int), d_sims float [n_layers, B, S - P] the similarities (only written on adaptive steps). */
+ * a HOST int), d_sims float [n_layers, B, S - P] the similarities (only written on adaptive steps).  Logits of response
+ * rows are defined on every step; logits of PROMPT rows only on steps that refresh the prompt (t mod k_prompt == 0): on the
+ * other steps nothing in the method reads the prompt rows of the residual stream, and they are not kept up to date. */
 int32_t sfs_forward_cached(sfs_session *session, const int32_t *d_tokens, int32_t B, int32_t S, int32_t P,
                            const sfs_state *d_state, const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
                            void *d_logits, int32_t logits_dtype, int32_t *d_sets, float *d_sims, int32_t *n_sel, void *stream);

@@ -154,20 +154,23 @@ static int32_t run_body(sfs_session *s, const int32_t *d_tokens, int32_t B, int3
 
 // ---- cached steps --------------------------------------------------------------------------------------
 // per-layer plans of the cached mode that do not depend on the number of recomputed rows
-static int32_t cache_plan(sfs_session *s, int32_t B, int32_t S)
+static int32_t cache_plan(sfs_session *s, int32_t B, int32_t S, int32_t P)
 {
     const sfs_model *m = s->model;
     const sfs_config &c = m->cfg;
     const int T = B * S, d = c.d_model, ff = c.d_ff;
-    if ((int)s->cache_plans.size() == c.n_layers && s->cache_B == B && s->cache_S == S) return SFS_OK;
+    if ((int)s->cache_plans.size() == c.n_layers && s->cache_B == B && s->cache_S == S && s->cache_P == P) return SFS_OK;
     s->cache_plans.assign(c.n_layers, CacheLayerPlans());
     s->gather_plans.clear();
     int32_t rc;
     for (int l = 0; l < c.n_layers; ++l) {
         CacheLayerPlans &cp = s->cache_plans[l];
         const void *wv[1] = {m->wv[l]};
-        // fresh values of every row, written transposed (every output column goes through the transposed store)
-        rc = gemm_plan_create(&cp.vproj, s->h, d, T, d, wv, 1, d, d, GEMM_STORE, s->attn, d, 0, 1.0f, s->vnew_t, T, 0, nullptr);
+        // fresh values of the candidate rows, written transposed (every output column goes through the transposed store): the
+        // response rows of a single sequence are one contiguous range; with several sequences every row is projected
+        const int v_first = (B == 1) ? P : 0, v_rows = (B == 1) ? S - P : T;
+        rc = gemm_plan_create(&cp.vproj, s->h + (size_t)v_first * d, d, v_rows, d, wv, 1, d, d, GEMM_STORE, s->attn, d, 0, 1.0f, s->vnew_t + v_first, T, 0,
+                              nullptr);
         if (rc != SFS_OK) return rc;
         const void *wo[1] = {m->wo[l]};
         rc = gemm_plan_create(&cp.o_store, s->attn, d, T, d, wo, 1, d, d, GEMM_STORE, s->Ac[l], d, 1, 1.0f, nullptr, 0, 0, nullptr);
@@ -199,12 +202,14 @@ static int32_t gather_plan(sfs_session *s, int32_t NR, int32_t T, std::vector<Ga
         const void *wo[1] = {m->wo[l]};
         rc = gemm_plan_create(&gp.o, s->attn, d, NR, d, wo, 1, d, d, GEMM_STORE, s->partial, d, 1, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
+        if ((rc = gemm_plan_enable_split(&gp.o, s->partial, kMaxSplits, nullptr)) != SFS_OK) return rc;   // few rows: K is split
         const void *gu[2] = {m->w_gate[l], m->w_up[l]};
         rc = gemm_plan_create(&gp.gate_up, s->hg, d, NR, d, gu, 2, ff, d, GEMM_SWIGLU, s->hid, ff, 0, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
         const void *wd[1] = {m->w_down[l]};
         rc = gemm_plan_create(&gp.down, s->hid, ff, NR, ff, wd, 1, d, ff, GEMM_STORE, s->partial, d, 1, 1.0f, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
+        if ((rc = gemm_plan_enable_split(&gp.down, s->partial, kMaxSplits, nullptr)) != SFS_OK) return rc;
     }
     auto ins = s->gather_plans.emplace(NR, std::move(v));
     *out = &ins.first->second;
@@ -229,7 +234,7 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
     SFS_REQUIRE(err != nullptr, SFS_ERR_OOM, "cannot allocate the device status word");
     int32_t rc;
     if ((rc = session_plan(s, B, S)) != SFS_OK) return rc;
-    if ((rc = cache_plan(s, B, S)) != SFS_OK) return rc;
+    if ((rc = cache_plan(s, B, S, P)) != SFS_OK) return rc;
     s->cache_B = B; s->cache_S = S; s->cache_P = P;
     const sfs_cache_params &cp = s->cache_params;
     const bool rp = (s->cache_t % cp.k_prompt) == 0, rr = (s->cache_t % cp.k_response) == 0;
@@ -241,8 +246,16 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
 
     if ((rc = timed_launch(s, SFS_K_EMBED, st, [&] { return launch_embed(d_tokens, m->tok_emb, s->x, T, d, c.vocab, st); })) != SFS_OK) return rc;
     const float *pend = nullptr;
+    // Rows whose residual stream this step keeps up to date: all of them, except that a single sequence whose prompt is not
+    // refreshed needs only its response rows (nothing reads the prompt rows of x or h then).
+    const int r_first = (B == 1 && !rp) ? P : 0, r_count = (B == 1 && !rp) ? L : T;
+    // tokens whose fresh values are compared with the cached ones: the response of a single sequence (from an even index), else all
+    const int sim_first = (B == 1) ? (P & ~1) : 0, sim_count = (B == 1) ? S - sim_first : T;
     auto norm_all = [&](const void *gain) {
-        return timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, pend, pend ? 1 : 0, 0, gain, s->h, nullptr, nullptr, T, d, c.rms_eps, st); });
+        return timed_launch(s, SFS_K_RMSNORM, st, [&] {
+            return launch_rmsnorm(s->x + (size_t)r_first * d, pend ? pend + (size_t)r_first * d : nullptr, pend ? 1 : 0, 0, gain,
+                                  s->h + (size_t)r_first * d, nullptr, nullptr, r_count, d, c.rms_eps, st);
+        });
     };
     if (rp && rr) {
         // everything is recomputed: the uncached layer pipeline, with the increments stored instead of added and K / V copied out
@@ -277,7 +290,7 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
                 const GatherLayerPlans &gp = (*gps)[l];
                 if (!rr && n_adapt > 0) {
                     if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(cl.vproj, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-                    if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_sim_partial(s->vnew_t, s->Vtc[l], T, d, T, s->sim_partial, st); })) != SFS_OK) return rc;
+                    if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_sim_partial(s->vnew_t, s->Vtc[l], T, d, sim_first, sim_count, T, s->sim_partial, st); })) != SFS_OK) return rc;
                 }
                 CacheSelectArgs a{};
                 a.partial = s->sim_partial; a.state = d_state; a.B = B; a.S = S; a.P = P; a.L = L; a.T = T;
@@ -291,7 +304,7 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
                 if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_kv(s->qk, 2 * d, d, s->vt, T, s->sel_rows, NR, d, s->Kc[l], s->Vtc[l], T, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch_queries(cl.attn, n_sel, d_active, err, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(gp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, s->sel_rows, NR, d, s->Ac[l], st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, gp.o.args.splits, gp.o.args.split_stride, s->sel_rows, NR, d, s->Ac[l], st); })) != SFS_OK) return rc;
             }
             pend = s->Ac[l];
             if ((rc = norm_all(m->mlp_norm[l])) != SFS_OK) return rc;
@@ -300,7 +313,7 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
                 if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_gather_rows_bf16(s->h, s->sel_rows, NR, d, s->hg, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(gp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(gp.down, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, s->sel_rows, NR, d, s->Fc[l], st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, gp.down.args.splits, gp.down.args.split_stride, s->sel_rows, NR, d, s->Fc[l], st); })) != SFS_OK) return rc;
             }
             pend = s->Fc[l];
         }

@@ -9,35 +9,46 @@ namespace {
 
 // grid (ceil(T / 64), kSimSlices), 256 threads: lane = two neighbouring tokens, warp = every 8th feature of the slice
 __global__ void __launch_bounds__(256)
-sim_partial_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b, long long ld, int d, int T,
+sim_partial_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b, long long ld, int d, int t_first, int t_end, int T,
                    float *__restrict__ partial)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int t0 = blockIdx.x * 64 + 2 * lane;
+    const int t0 = t_first + blockIdx.x * 64 + 2 * lane;             // t_first is even: 4-byte loads of two tokens stay aligned
     const int per = (d + kSimSlices - 1) / kSimSlices;
     const int f0 = blockIdx.y * per, f1 = min(d, f0 + per);
     float acc[6] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-    if (t0 < T) {
-        for (int f = f0 + warp; f < f1; f += 8) {
-            const uint32_t wa = *reinterpret_cast<const uint32_t *>(a + (long long)f * ld + t0);
-            const uint32_t wb = *reinterpret_cast<const uint32_t *>(b + (long long)f * ld + t0);
+    if (t0 < t_end) {
+        auto term = [&](uint32_t wa, uint32_t wb) {
             const float a0 = bf16_bits_to_f32(wa & 0xFFFFu), a1 = bf16_bits_to_f32(wa >> 16);
             const float b0 = bf16_bits_to_f32(wb & 0xFFFFu), b1 = bf16_bits_to_f32(wb >> 16);
             acc[0] = fmaf(a0, b0, acc[0]); acc[1] = fmaf(a0, a0, acc[1]); acc[2] = fmaf(b0, b0, acc[2]);
             acc[3] = fmaf(a1, b1, acc[3]); acc[4] = fmaf(a1, a1, acc[4]); acc[5] = fmaf(b1, b1, acc[5]);
+        };
+        int f = f0 + warp;
+        for (; f + 24 < f1; f += 32) {                               // four features per round: eight loads in flight
+            uint32_t wa[4], wb[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                wa[u] = *reinterpret_cast<const uint32_t *>(a + (long long)(f + 8 * u) * ld + t0);
+                wb[u] = *reinterpret_cast<const uint32_t *>(b + (long long)(f + 8 * u) * ld + t0);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) term(wa[u], wb[u]);           // same feature order as the plain loop
         }
+        for (; f < f1; f += 8)
+            term(*reinterpret_cast<const uint32_t *>(a + (long long)f * ld + t0), *reinterpret_cast<const uint32_t *>(b + (long long)f * ld + t0));
     }
     __shared__ float s[8][32][6];
 #pragma unroll
     for (int i = 0; i < 6; ++i) s[warp][lane][i] = acc[i];
     __syncthreads();
-    if (warp == 0 && t0 < T) {
+    if (warp == 0 && t0 < t_end) {
         float r[6];
 #pragma unroll
         for (int i = 0; i < 6; ++i) { r[i] = s[0][lane][i]; for (int w = 1; w < 8; ++w) r[i] += s[w][lane][i]; }   // fixed order
         float *o = partial + ((long long)blockIdx.y * T + t0) * 3;
         o[0] = r[0]; o[1] = r[1]; o[2] = r[2];
-        if (t0 + 1 < T) { o[3] = r[3]; o[4] = r[4]; o[5] = r[5]; }
+        if (t0 + 1 < t_end) { o[3] = r[3]; o[4] = r[4]; o[5] = r[5]; }
     }
 }
 
@@ -47,7 +58,7 @@ __device__ __forceinline__ uint32_t float_order_key(float f) {       // monotone
 }
 
 // one CTA per sequence; dynamic shared memory: u64 keys[L], u8 chosen[L]
-__global__ void __launch_bounds__(256) cache_select_kernel(CacheSelectArgs a)
+__global__ void __launch_bounds__(1024) cache_select_kernel(CacheSelectArgs a)
 {
     extern __shared__ unsigned long long s_key[];
     const int b = blockIdx.x, tid = threadIdx.x, L = a.L, P = a.P, S = a.S;
@@ -116,41 +127,61 @@ __global__ void gather_rows_bf16_kernel(const uint4 *__restrict__ src, const int
     for (int c = threadIdx.x; c < chunks; c += blockDim.x) o[c] = s[c];
 }
 
-__global__ void scatter_rows_f32_kernel(const float4 *__restrict__ src, const int32_t *__restrict__ rows, int chunks, float4 *__restrict__ dst)
+__global__ void scatter_rows_f32_kernel(const float4 *__restrict__ src, int n_slabs, long long slab_chunks, const int32_t *__restrict__ rows,
+                                        int chunks, float4 *__restrict__ dst)
 {
     const int j = blockIdx.x;
     const float4 *s = src + (long long)j * chunks;
     float4 *o = dst + (long long)rows[j] * chunks;
-    for (int c = threadIdx.x; c < chunks; c += blockDim.x) o[c] = s[c];
+    for (int c = blockIdx.y * blockDim.x + threadIdx.x; c < chunks; c += gridDim.y * blockDim.x) {
+        float4 v = s[c];
+        for (int k = 1; k < n_slabs; ++k) {                  // split-K partial products, added in slab order
+            const float4 p = s[(long long)k * slab_chunks + c];
+            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+        }
+        o[c] = v;
+    }
 }
 
-// blockIdx.x = compact row j: copies its K row; blockIdx.y selects a slab of features for the V^T columns
-__global__ void scatter_kv_kernel(const __nv_bfloat16 *__restrict__ qk, long long ld_src, int col0,
-                                  const __nv_bfloat16 *__restrict__ vt_src, long long ld_vt_src, const int32_t *__restrict__ rows,
-                                  int d, __nv_bfloat16 *__restrict__ k_dst, __nv_bfloat16 *__restrict__ vt_dst, long long ld_vt_dst)
+// K rows: block j copies compact row j to its token row
+__global__ void scatter_k_kernel(const __nv_bfloat16 *__restrict__ qk, long long ld_src, int col0, const int32_t *__restrict__ rows,
+                                 int d, __nv_bfloat16 *__restrict__ k_dst)
 {
     const int j = blockIdx.x;
-    const int r = rows[j];
     const uint4 *s = reinterpret_cast<const uint4 *>(qk + (long long)j * ld_src + col0);
-    uint4 *o = reinterpret_cast<uint4 *>(k_dst + (long long)r * d);
+    uint4 *o = reinterpret_cast<uint4 *>(k_dst + (long long)rows[j] * d);
     for (int c = threadIdx.x; c < d / 8; c += blockDim.x) o[c] = s[c];
-    for (int f = threadIdx.x; f < d; f += blockDim.x) vt_dst[(long long)f * ld_vt_dst + r] = vt_src[(long long)f * ld_vt_src + j];
+}
+
+// V^T columns: a block owns 8 features; compact rows run fastest over the threads, so the reads are contiguous
+__global__ void scatter_vt_kernel(const __nv_bfloat16 *__restrict__ vt_src, long long ld_vt_src, const int32_t *__restrict__ rows, int n_rows,
+                                  int d, __nv_bfloat16 *__restrict__ vt_dst, long long ld_vt_dst)
+{
+    const int f0 = blockIdx.x * 8;
+    for (int idx = threadIdx.x; idx < 8 * n_rows; idx += blockDim.x) {
+        const int f = f0 + idx / n_rows, j = idx - (idx / n_rows) * n_rows;
+        if (f < d) vt_dst[(long long)f * ld_vt_dst + rows[j]] = vt_src[(long long)f * ld_vt_src + j];
+    }
 }
 
 }  // namespace
 
-int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld, int d, int T, float *partial, cudaStream_t s)
+int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld, int d, int t_first, int t_count, int T, float *partial,
+                           cudaStream_t s)
 {
-    dim3 grid((unsigned)((T + 63) / 64), kSimSlices, 1);
+    if (t_count <= 0) return SFS_OK;
+    SFS_REQUIRE((t_first % 2) == 0 && (ld % 2) == 0, SFS_ERR_INVALID_ARG, "similarity: first token and row stride must be even");
+    dim3 grid((unsigned)((t_count + 63) / 64), kSimSlices, 1);
     sim_partial_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(vnew_t), reinterpret_cast<const __nv_bfloat16 *>(vold_t),
-                                            ld, d, T, partial);
+                                            ld, d, t_first, t_first + t_count, T, partial);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }
 
 int32_t launch_cache_select(const CacheSelectArgs &a, cudaStream_t s)
 {
-    cache_select_kernel<<<a.B, 256, (size_t)a.L * 9 + 16, s>>>(a);
+    const int threads = a.L >= 512 ? 1024 : (a.L > 256 ? 512 : 256);         // the ranking is O(L^2 / threads)
+    cache_select_kernel<<<a.B, threads, (size_t)a.L * 9 + 16, s>>>(a);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }
@@ -163,10 +194,12 @@ int32_t launch_gather_rows_bf16(const void *src, const int32_t *rows, int n_rows
     return SFS_OK;
 }
 
-int32_t launch_scatter_rows_f32(const float *src, const int32_t *rows, int n_rows, int d, float *dst, cudaStream_t s)
+int32_t launch_scatter_rows_f32(const float *src, int n_slabs, long long slab_stride, const int32_t *rows, int n_rows, int d, float *dst,
+                                cudaStream_t s)
 {
     if (n_rows <= 0) return SFS_OK;
-    scatter_rows_f32_kernel<<<n_rows, 128, 0, s>>>(reinterpret_cast<const float4 *>(src), rows, d / 4, reinterpret_cast<float4 *>(dst));
+    scatter_rows_f32_kernel<<<dim3((unsigned)n_rows, 4, 1), 256, 0, s>>>(reinterpret_cast<const float4 *>(src), n_slabs < 1 ? 1 : n_slabs, slab_stride / 4, rows, d / 4,
+                                                   reinterpret_cast<float4 *>(dst));
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }
@@ -175,9 +208,11 @@ int32_t launch_scatter_kv(const void *qk_src, long long ld_src, int col0, const 
                           const int32_t *rows, int n_rows, int d, void *k_dst, void *vt_dst, long long ld_vt_dst, cudaStream_t s)
 {
     if (n_rows <= 0) return SFS_OK;
-    scatter_kv_kernel<<<n_rows, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(qk_src), ld_src, col0,
-                                             reinterpret_cast<const __nv_bfloat16 *>(vt_src), ld_vt_src, rows, d,
-                                             reinterpret_cast<__nv_bfloat16 *>(k_dst), reinterpret_cast<__nv_bfloat16 *>(vt_dst), ld_vt_dst);
+    scatter_k_kernel<<<n_rows, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(qk_src), ld_src, col0, rows, d,
+                                            reinterpret_cast<__nv_bfloat16 *>(k_dst));
+    SFS_LAUNCH_CHECK();
+    scatter_vt_kernel<<<(d + 7) / 8, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(vt_src), ld_vt_src, rows, n_rows, d,
+                                                  reinterpret_cast<__nv_bfloat16 *>(vt_dst), ld_vt_dst);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }

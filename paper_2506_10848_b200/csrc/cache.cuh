@@ -4,11 +4,13 @@
 
 namespace sfs {
 
-constexpr int kSimSlices = 8;          // the feature dimension is cut into this many slices for the similarity sums
+constexpr int kSimSlices = 32;         // the feature dimension is cut into this many slices for the similarity sums
 
-// partial[slice][t][0..2] = sum over the slice's features of (v_new * v_old, v_new^2, v_old^2) for token t;
-// both operands are feature-major bf16 [d, T] with ld elements between feature rows.
-int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld, int d, int T, float *partial, cudaStream_t s);
+// partial[slice][t][0..2] = sum over the slice's features of (v_new * v_old, v_new^2, v_old^2) for the tokens
+// t_first <= t < t_first + t_count (t_first even); both operands are feature-major bf16 [d, T] with ld elements between
+// feature rows; partial is [kSimSlices, T, 3] whatever the token range.
+int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld, int d, int t_first, int t_count, int T, float *partial,
+                           cudaStream_t s);
 
 struct CacheSelectArgs {
     const float *partial;              // [kSimSlices, T, 3]
@@ -27,8 +29,10 @@ struct CacheSelectArgs {
 int32_t launch_cache_select(const CacheSelectArgs &a, cudaStream_t s);
 
 int32_t launch_gather_rows_bf16(const void *src, const int32_t *rows, int n_rows, int d, void *dst, cudaStream_t s);
-// dst[rows[j], :] = src[j, :]   (fp32 rows of d elements)
-int32_t launch_scatter_rows_f32(const float *src, const int32_t *rows, int n_rows, int d, float *dst, cudaStream_t s);
+// dst[rows[j], :] = sum over k < n_slabs of src[k * slab_stride + j * d + :]   (fp32 rows of d elements; slabs = the partial
+// products of a split-K projection, added in slab order)
+int32_t launch_scatter_rows_f32(const float *src, int n_slabs, long long slab_stride, const int32_t *rows, int n_rows, int d, float *dst,
+                                cudaStream_t s);
 // K rows: dst[rows[j], 0:d] = src[j, col0 : col0 + d] (bf16, src ld = ld_src);  V columns: dst_t[f, rows[j]] = src_t[f, j]
 int32_t launch_scatter_kv(const void *qk_src, long long ld_src, int col0, const void *vt_src, long long ld_vt_src,
                           const int32_t *rows, int n_rows, int d, void *k_dst, void *vt_dst, long long ld_vt_dst, cudaStream_t s);

@@ -522,7 +522,8 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
 int32_t gemm_plan_enable_split(GemmPlan *p, float *ws, int32_t max_splits, const GemmTune *tune)
 {
     GemmArgs &g = p->args;
-    if (g.mode != GEMM_RESIDUAL_F32 || ws == nullptr || max_splits < 2) return SFS_OK;
+    const bool f32_out = g.mode == GEMM_RESIDUAL_F32 || (g.mode == GEMM_STORE && g.out_f32 && g.vt == nullptr);
+    if (!f32_out || ws == nullptr || max_splits < 2) return SFS_OK;
     int mb = g.mb, bn = g.bn, sp = 1;
     pick_tile(g.M, g.K, g.mode, p->n_maps, p->n_per_map, num_sms() / 2, max_splits, &mb, &bn, &sp);
     if (tune) {
