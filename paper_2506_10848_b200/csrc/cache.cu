@@ -77,10 +77,15 @@ __global__ void __launch_bounds__(1024) cache_select_kernel(CacheSelectArgs a)
         for (int i = tid; i < L; i += blockDim.x) {
             float dot = 0.f, na = 0.f, nb = 0.f;
             const long long t = (long long)b * S + P + i;
-            for (int sl = 0; sl < kSimSlices; ++sl) {                // fixed order
-                const float *p = a.partial + ((long long)sl * a.T + t) * 3;
-                dot += p[0]; na += p[1]; nb += p[2];
+            const float *__restrict__ part = a.partial;
+            float pd[kSimSlices], pa[kSimSlices], pb[kSimSlices];
+#pragma unroll
+            for (int sl = 0; sl < kSimSlices; ++sl) {                // all loads first: one latency, not kSimSlices of them
+                const float *p = part + ((long long)sl * a.T + t) * 3;
+                pd[sl] = __ldg(p); pa[sl] = __ldg(p + 1); pb[sl] = __ldg(p + 2);
             }
+#pragma unroll
+            for (int sl = 0; sl < kSimSlices; ++sl) { dot += pd[sl]; na += pa[sl]; nb += pb[sl]; }   // fixed order
             const float den = __fmul_rn(__fsqrt_rn(na), __fsqrt_rn(nb));
             const float sim = den > 0.f ? __fdiv_rn(dot, den) : 0.f;
             if (a.sims_dump) a.sims_dump[(long long)b * L + i] = sim;
