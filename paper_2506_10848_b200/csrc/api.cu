@@ -283,9 +283,17 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
     } else {
         std::vector<GatherLayerPlans> *gps = nullptr;
         if (NR > 0 && (rc = gather_plan(s, NR, T, &gps)) != SFS_OK) return rc;
+        // Here the attention increment of a layer stays pending through its MLP branch: the MLP norm reads x + A_l for the
+        // recomputed rows only (straight into the compact buffer), and the next layer's first norm folds A_l and F_l together.
+        const long long inc_stride = (long long)s->max_batch * s->max_seq * d;     // A_l -> F_l
+        int n_pend = 0;
         for (int l = 0; l < c.n_layers; ++l) {
             const CacheLayerPlans &cl = s->cache_plans[l];
-            if ((rc = norm_all(m->attn_norm[l])) != SFS_OK) return rc;
+            rc = timed_launch(s, SFS_K_RMSNORM, st, [&] {
+                return launch_rmsnorm(s->x + (size_t)r_first * d, pend ? pend + (size_t)r_first * d : nullptr, n_pend, inc_stride, m->attn_norm[l],
+                                      s->h + (size_t)r_first * d, nullptr, nullptr, r_count, d, c.rms_eps, st);
+            });
+            if (rc != SFS_OK) return rc;
             if (NR > 0) {
                 const GatherLayerPlans &gp = (*gps)[l];
                 if (!rr && n_adapt > 0) {
@@ -306,17 +314,21 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
                 if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(gp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, gp.o.args.splits, gp.o.args.split_stride, s->sel_rows, NR, d, s->Ac[l], st); })) != SFS_OK) return rc;
             }
-            pend = s->Ac[l];
-            if ((rc = norm_all(m->mlp_norm[l])) != SFS_OK) return rc;
+            pend = s->Ac[l]; n_pend = 2;
             if (NR > 0) {
                 const GatherLayerPlans &gp = (*gps)[l];
-                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_gather_rows_bf16(s->h, s->sel_rows, NR, d, s->hg, st); })) != SFS_OK) return rc;
+                rc = timed_launch(s, SFS_K_RMSNORM, st, [&] {
+                    return launch_rmsnorm(s->x, s->Ac[l], 1, 0, m->mlp_norm[l], s->hg, s->sel_rows, nullptr, NR, d, c.rms_eps, st);
+                });
+                if (rc != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(gp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_DOWN, st, [&] { return gemm_launch(gp.down, nullptr, d_active, err, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, gp.down.args.splits, gp.down.args.split_stride, s->sel_rows, NR, d, s->Fc[l], st); })) != SFS_OK) return rc;
             }
-            pend = s->Fc[l];
         }
+        s->pending_ptr = pend; s->pending_n = pend ? n_pend : 0; s->pending_stride = inc_stride;
+        s->cache_t++;
+        return SFS_OK;
     }
     s->pending_ptr = pend; s->pending_n = pend ? 1 : 0; s->pending_stride = 0;
     s->cache_t++;
@@ -584,8 +596,9 @@ int32_t sfs_cache_enable(sfs_session *s, const sfs_cache_params *p)
         for (int l = 0; l < c.n_layers; ++l) {
             if ((rc = dev_alloc(s, &s->Kc[l], T * d, true)) != SFS_OK) return rc;
             if ((rc = dev_alloc(s, &s->Vtc[l], T * d, true)) != SFS_OK) return rc;
-            if ((rc = dev_alloc(s, &s->Ac[l], T * d, true)) != SFS_OK) return rc;
-            if ((rc = dev_alloc(s, &s->Fc[l], T * d, true)) != SFS_OK) return rc;
+            // the two increments of a layer lie T * d floats apart, so one norm can fold both as two slabs
+            if ((rc = dev_alloc(s, &s->Ac[l], 2 * T * d, true)) != SFS_OK) return rc;
+            s->Fc[l] = s->Ac[l] + T * d;
         }
         if ((rc = dev_alloc(s, &s->hg, T * d, true)) != SFS_OK) return rc;
         if ((rc = dev_alloc(s, &s->vnew_t, T * d, true)) != SFS_OK) return rc;
