@@ -44,17 +44,33 @@ rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ partial, int n_p
         float4 *xr = reinterpret_cast<float4 *>(x + src * d);
         const float4 *pr = reinterpret_cast<const float4 *>(partial + src * d);
         const long long pstride4 = partial_stride / 4;
-        float4 keep[kNormRegChunks];
-        float ss = 0.f;
-        int k = 0;
-        for (int c = threadIdx.x; c < chunks; c += kNormThreads, ++k) {
+        auto load = [&](int c) {                              // x + the partial products, slab by slab
             float4 v = xr[c];
             for (int s = 0; s < n_partial; ++s) {
                 const float4 p = pr[(long long)s * pstride4 + c];
                 v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
             }
+            return v;
+        };
+        // the first kNormRegChunks chunks of a thread stay in registers (statically indexed); longer rows re-read the rest
+        float4 keep[kNormRegChunks];
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < kNormRegChunks; ++k) {
+            const int c = threadIdx.x + k * kNormThreads;
+            keep[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c < chunks) keep[k] = load(c);
+        }
+#pragma unroll
+        for (int k = 0; k < kNormRegChunks; ++k) {
+            const int c = threadIdx.x + k * kNormThreads;
+            const float4 v = keep[k];
+            if (c < chunks && n_partial > 0 && rows == nullptr) xr[c] = v;
+            ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+        for (int c = threadIdx.x + kNormRegChunks * kNormThreads; c < chunks; c += kNormThreads) {
+            const float4 v = load(c);
             if (n_partial > 0 && rows == nullptr) xr[c] = v;
-            if (k < kNormRegChunks) keep[k] = v;
             ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         }
         ss = warp_sum(ss);
@@ -66,22 +82,21 @@ rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ partial, int n_p
         const float inv = rsqrtf(tot / (float)d + eps);
         const uint2 *gp = reinterpret_cast<const uint2 *>(gain);
         uint2 *hp = reinterpret_cast<uint2 *>(h + (long long)r * d);
-        k = 0;
-        for (int c = threadIdx.x; c < chunks; c += kNormThreads, ++k) {
-            float4 v;
-            if (k < kNormRegChunks) v = keep[k];
-            else {                                           // long rows: rebuild the value the first pass saw
-                v = xr[c];
-                if (rows != nullptr)
-                    for (int s = 0; s < n_partial; ++s) {
-                        const float4 p = pr[(long long)s * pstride4 + c];
-                        v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-                    }
-            }
+        auto emit = [&](int c, const float4 &v) {
             const uint2 g = gp[c];
             __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * inv * bf16_bits_to_f32(g.x & 0xFFFFu), v.y * inv * bf16_bits_to_f32(g.x >> 16));
             __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * inv * bf16_bits_to_f32(g.y & 0xFFFFu), v.w * inv * bf16_bits_to_f32(g.y >> 16));
             hp[c] = make_uint2(*reinterpret_cast<uint32_t *>(&o0), *reinterpret_cast<uint32_t *>(&o1));
+        };
+#pragma unroll
+        for (int k = 0; k < kNormRegChunks; ++k) {
+            const int c = threadIdx.x + k * kNormThreads;
+            if (c < chunks) emit(c, keep[k]);
+        }
+        for (int c = threadIdx.x + kNormRegChunks * kNormThreads; c < chunks; c += kNormThreads) {
+            // long rows: rebuild the value the first pass saw (x already holds it when it was written back)
+            const float4 v = (rows == nullptr && n_partial > 0) ? xr[c] : load(c);
+            emit(c, v);
         }
         __syncthreads();
     }
