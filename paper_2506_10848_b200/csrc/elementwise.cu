@@ -118,12 +118,14 @@ __global__ void rope_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int T,
 {
     // one thread handles 8 consecutive j of one (token, q-or-k, head)
     const int half = dh / 2, groups = half / 8;
-    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long total = (long long)T * 2 * n_heads * groups;
+    const unsigned idx = blockIdx.x * blockDim.x + threadIdx.x;   // the launcher checks that the item count fits 31 bits
+    const unsigned total = (unsigned)T * 2u * (unsigned)n_heads * (unsigned)groups;
     if (idx >= total) return;
-    const int g = (int)(idx % groups);
-    const int hh = (int)((idx / groups) % (2 * n_heads));      // q heads then k heads: contiguous columns
-    const int t = (int)(idx / ((long long)groups * 2 * n_heads));
+    const unsigned per_token = (unsigned)groups * 2u * (unsigned)n_heads;
+    const int t = (int)(idx / per_token);
+    const unsigned rem = idx - (unsigned)t * per_token;
+    const int hh = (int)(rem / (unsigned)groups);              // q heads then k heads: contiguous columns
+    const int g = (int)(rem - (unsigned)hh * (unsigned)groups);
     const int pos = (rows ? rows[t] : t) % S;              // compact rows carry the token index they came from
     __nv_bfloat16 *base = qk + (long long)t * ld + (long long)hh * dh + g * 8;
     uint4 lo = *reinterpret_cast<uint4 *>(base), hi = *reinterpret_cast<uint4 *>(base + half);
@@ -180,6 +182,7 @@ int32_t launch_rope_table(float2 *table, int positions, int head_dim, float thet
 int32_t launch_rope(void *qk, int64_t ld, int T, int S, int n_heads, int head_dim, const float2 *table, const int32_t *rows, cudaStream_t s)
 {
     const long long total = (long long)T * 2 * n_heads * (head_dim / 16);
+    SFS_REQUIRE(total < (1LL << 31), SFS_ERR_INVALID_ARG, "rope: %lld items do not fit a 32-bit index", total);
     rope_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<__nv_bfloat16 *>(qk), ld, T, S, n_heads, head_dim, table, rows);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
