@@ -7,7 +7,7 @@
 namespace sfs {
 namespace {
 
-// grid (ceil(T / 64), kSimSlices), 256 threads: lane = two neighbouring tokens, warp = every 8th feature of the slice
+// grid (ceil(tokens / 64), kSimSlices), 256 threads: lane = two neighbouring tokens, warp = every 8th feature of the slice
 __global__ void __launch_bounds__(256)
 sim_partial_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b, long long ld, int d, int t_first, int t_end, int T,
                    float *__restrict__ partial)

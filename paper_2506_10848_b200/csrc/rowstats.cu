@@ -1,11 +1,13 @@
 // Row statistics of the sampling epilogue (paper Section 3.1): per logits row the greedy token
 // r_hat = argmax_v x_v and the canonical fixed-point softmax denominator S_q (c = 2^28 / S_q).
 //
-// Fast path (bf16 logits): a thread-block cluster owns one row.  Every thread keeps its 16-byte chunks of
-// the row in registers, so HBM is read exactly once: pass 1 (registers) finds the exact row maximum, the
-// cluster exchanges it through distributed shared memory, pass 2 (registers again) evaluates the
-// fixed-point exponentials with packed f32x2 arithmetic and sums them as integers.  Integer sums make the
-// result independent of how the row is split over threads, warps and CTAs.
+// Fast paths (bf16 logits): a thread-block cluster owns one row and HBM is read exactly once.  Pass 1 finds the exact row
+// maximum, the CTAs push their slice maxima to each other through distributed shared memory (one cluster barrier), pass 2
+// evaluates the fixed-point exponentials with packed f32x2 arithmetic and sums them as integers; sums and first-maximum
+// candidates reach rank 0 by remote shared-memory atomics.  Integer sums make the result independent of how the row is
+// split over threads, warps and CTAs.  Rows of 128 KB and more are staged: each of 8 CTAs brings its contiguous slice into
+// shared memory with one bulk asynchronous copy (no registers tied up in flight, seven CTAs per SM); shorter rows stay in
+// registers (every thread keeps its 16-byte chunks between the passes).
 //
 // Generic path (bf16 or fp32, any vocabulary size or stride): one CTA per row, two sweeps over global memory.
 #include "sfs_common.cuh"
