@@ -62,6 +62,10 @@ def test_logits_of_sampled_rows_match_the_oracle_at_the_8b_shape(model8b):
         sfs.sfs_forward(session, tok.to(DEV), B, S, d_rows, None, len(rows), lg, sfs.LOGITS_F32)
         sfs.sfs_check_device_status()
         got = lg.cpu().double().numpy()
+        # the same call again gives the same bits: split-K slabs, the attention's exchanges and the residual adds have a fixed order
+        lg2 = torch.zeros_like(lg)
+        sfs.sfs_forward(session, tok.to(DEV), B, S, d_rows, None, len(rows), lg2, sfs.LOGITS_F32)
+        assert torch.equal(lg, lg2)
     finally:
         sfs.sfs_session_destroy(session)
     conv = lambda t: t.detach().to("cpu").to(torch.float32).numpy()
