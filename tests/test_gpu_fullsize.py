@@ -199,3 +199,52 @@ def test_cached_steps_match_the_oracle_at_the_8b_shape_under_the_same_schedule(m
     finally:
         sfs.sfs_cache_enable(session, 1, 1, 0.0, off=True)
         sfs.sfs_session_destroy(session)
+
+
+@pytest.mark.parametrize("B,P,L,n_steps,seed", [(1, 256, 256, 5, 2), (8, 512, 256, 3, 4)])
+def test_first_steps_of_the_8b_loop_are_reproduced_by_the_oracle_scheduler(model8b, B, P, L, n_steps, seed):
+    """The benchmark's own configurations (batch 1, 256 + 256; batch 8, 512 + 256): the device loop runs step by step with its
+    logits dumped; the oracle's row statistics and scheduler, fed those logits, must give the same row lists, decisions and
+    tokens bit for bit, every sequence with its own state."""
+    from oracle import rowstats as RS
+    from oracle.scheduler import SlowFastParams, SlowFastState, rows_needed, slowfast_step
+    shape, w, model = model8b
+    S = P + L
+    po = SlowFastParams()
+    pg = sfs.Params.default(**{k: getattr(po, k) for k in ("tau_min_conf", "tau_high_conf", "sigma2_stable", "k_max", "w_hist", "k_slow",
+                                                           "k_fast", "max_steps", "min_high_count")})
+    prompt = W.prompt_ids(B, P, shape.vocab - 2, seed=seed)
+    session = sfs.sfs_session_create(model, B, S)
+    try:
+        trace = torch.zeros((n_steps, B, sfs.TRACE_INTS), dtype=torch.int32, device=DEV)
+        dump = torch.zeros((B * L, shape.vocab), dtype=torch.bfloat16, device=DEV)
+        rows_d = torch.zeros(B * L, dtype=torch.int32, device=DEV)
+        nrows_d = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sfs.sfs_generate_begin(session, prompt.to(DEV), B, P, L, pg)
+        st = [SlowFastState.fresh(L, po) for _ in range(B)]
+        y = [dict() for _ in range(B)]
+        for step in range(n_steps):
+            sfs.sfs_generate_steps(session, 1, trace, n_steps, dump, rows_d, nrows_d)
+            torch.cuda.synchronize()
+            need = [(b, i) for b in range(B) for i in rows_needed(st[b])]
+            n = int(nrows_d.item())
+            assert rows_d[:n].tolist() == [b * S + P + i for (b, i) in need], step
+            stats = RS.row_stats(W.bf16_bits(dump[:n].cpu()))
+            for b in range(B):
+                idx = {i: j for j, (bb, i) in enumerate(need) if bb == b}
+                rec = slowfast_step(st[b], {i: int(stats["argmax"][j]) for i, j in idx.items()},
+                                    {i: int(stats["sq"][j]) for i, j in idx.items()}, po)
+                for i, t in zip(rec.positions, rec.tokens):
+                    y[b][i] = t
+                assert trace[step, b].tolist()[:6] == [rec.phase, rec.s, rec.hi, rec.e_cand, rec.stable, len(rec.positions)], (step, b, rec)
+        out = torch.zeros((B, S), dtype=torch.int32, device=DEV)
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+        sfs.sfs_generate_end(session, out, state)
+        sfs.sfs_check_device_status()
+        f = sfs.STATE_FIELDS.index
+        for b in range(B):
+            o = out[b, P:].cpu().tolist()
+            assert len(y[b]) >= n_steps and all(o[i] == t for i, t in y[b].items()), b
+            assert int(state[b, f("n_masked")]) == L - len(y[b]) and int(state[b, f("steps_done")]) == n_steps
+    finally:
+        sfs.sfs_session_destroy(session)
