@@ -201,14 +201,20 @@ def test_cached_steps_match_the_oracle_at_the_8b_shape_under_the_same_schedule(m
         sfs.sfs_session_destroy(session)
 
 
-@pytest.mark.parametrize("B,P,L,n_steps,seed", [(1, 256, 256, 5, 2), (8, 512, 256, 3, 4)])
-def test_first_steps_of_the_8b_loop_are_reproduced_by_the_oracle_scheduler(model8b, B, P, L, n_steps, seed):
+@pytest.mark.parametrize("B,P,L,n_steps,seed,scale", [(1, 256, 256, 5, 2, None), (8, 512, 256, 3, 4, None), (2, 256, 256, 8, 2, 300.0)])
+def test_first_steps_of_the_8b_loop_are_reproduced_by_the_oracle_scheduler(model8b, B, P, L, n_steps, seed, scale):
     """The benchmark's own configurations (batch 1, 256 + 256; batch 8, 512 + 256): the device loop runs step by step with its
     logits dumped; the oracle's row statistics and scheduler, fed those logits, must give the same row lists, decisions and
-    tokens bit for bit, every sequence with its own state."""
+    tokens bit for bit, every sequence with its own state.  With random-init weights every max-prob is ~1e-3 and each step
+    unmasks one token; the third case multiplies the logits by 300 (same weights, another logit scale), so that both thresholds
+    fire and fast steps with many tokens run at the full shape."""
     from oracle import rowstats as RS
     from oracle.scheduler import SlowFastParams, SlowFastState, rows_needed, slowfast_step
     shape, w, model = model8b
+    own_model = None
+    if scale is not None:                                      # the same device weights under another logit scale
+        dct = shape.asdict(); dct["logit_scale"] = scale
+        own_model = model = sfs.Model(W.Shape(**dct), w)
     S = P + L
     po = SlowFastParams()
     pg = sfs.Params.default(**{k: getattr(po, k) for k in ("tau_min_conf", "tau_high_conf", "sigma2_stable", "k_max", "w_hist", "k_slow",
@@ -223,7 +229,10 @@ def test_first_steps_of_the_8b_loop_are_reproduced_by_the_oracle_scheduler(model
         sfs.sfs_generate_begin(session, prompt.to(DEV), B, P, L, pg)
         st = [SlowFastState.fresh(L, po) for _ in range(B)]
         y = [dict() for _ in range(B)]
+        done_steps = [0] * B
         for step in range(n_steps):
+            if all(s_.done for s_ in st):
+                break
             sfs.sfs_generate_steps(session, 1, trace, n_steps, dump, rows_d, nrows_d)
             torch.cuda.synchronize()
             need = [(b, i) for b in range(B) for i in rows_needed(st[b])]
@@ -231,6 +240,9 @@ def test_first_steps_of_the_8b_loop_are_reproduced_by_the_oracle_scheduler(model
             assert rows_d[:n].tolist() == [b * S + P + i for (b, i) in need], step
             stats = RS.row_stats(W.bf16_bits(dump[:n].cpu()))
             for b in range(B):
+                if st[b].done:
+                    continue
+                done_steps[b] += 1
                 idx = {i: j for j, (bb, i) in enumerate(need) if bb == b}
                 rec = slowfast_step(st[b], {i: int(stats["argmax"][j]) for i, j in idx.items()},
                                     {i: int(stats["sq"][j]) for i, j in idx.items()}, po)
@@ -244,7 +256,12 @@ def test_first_steps_of_the_8b_loop_are_reproduced_by_the_oracle_scheduler(model
         f = sfs.STATE_FIELDS.index
         for b in range(B):
             o = out[b, P:].cpu().tolist()
-            assert len(y[b]) >= n_steps and all(o[i] == t for i, t in y[b].items()), b
-            assert int(state[b, f("n_masked")]) == L - len(y[b]) and int(state[b, f("steps_done")]) == n_steps
+            assert len(y[b]) >= done_steps[b] and all(o[i] == t for i, t in y[b].items()), b
+            assert int(state[b, f("n_masked")]) == L - len(y[b]) and int(state[b, f("steps_done")]) == done_steps[b]
+        print(f"B={B} scale={scale}: tokens unmasked per sequence {[len(v) for v in y]} in {done_steps} steps")
+        if scale is not None:
+            assert max(len(v) for v in y) > max(done_steps)      # parallel unmasking happened
     finally:
         sfs.sfs_session_destroy(session)
+        if own_model is not None:
+            own_model.close()
