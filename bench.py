@@ -310,8 +310,10 @@ def run_extras(torch, sfs, W, model, shape, dev, peaks, weights=None):
     ms = sum(ts) / len(ts)
     g_fl, a_fl, h_fl = step_flops(shape, B * (P + L), P + L, B * L)
     roof = max((g_fl + a_fl + h_fl) / (peaks["bf16_tflops"] * 1e12), step_bytes(shape, B * (P + L), B * L) / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    roof_sus = max((g_fl + a_fl + h_fl) / (peaks["bf16_tflops_sustained"] * 1e12), step_bytes(shape, B * (P + L), B * L) / (peaks["hbm_gbs"] * 1e9)) * 1e3
     out["batch8_512_256"] = {"workload": "8B shape, batch 8, prompt 512 + 256 masked, seed 4", "ms_per_step": ms, "tokens_per_s": B / (ms * 1e-3),
                              "step_roofline_ms": roof, "step_roofline_frac": roof / ms,
+                             "step_roofline_ms_sustained_peak": roof_sus, "step_roofline_frac_sustained_peak": roof_sus / ms,
                              "note": "one token per sequence and step with random-init logits"}
     sfs.sfs_session_destroy(session)
     torch.cuda.empty_cache()
@@ -483,6 +485,7 @@ def main():
     ms_step = ms / K
     g_fl, a_fl, h_fl = step_flops(shape, res["T"], res["S"], res["head_rows"])
     step_roof_ms = max((g_fl + a_fl + h_fl) / (peaks["bf16_tflops"] * 1e12), step_bytes(shape, res["T"], res["head_rows"]) / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    step_roof_sus_ms = max((g_fl + a_fl + h_fl) / (peaks["bf16_tflops_sustained"] * 1e12), step_bytes(shape, res["T"], res["head_rows"]) / (peaks["hbm_gbs"] * 1e9)) * 1e3
     roofline = {"bound": "tensor", "achieved": res["gemm_tflops"], "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": (res["gemm_tflops"] / peaks["bf16_tflops_sustained"]) if res["gemm_tflops"] else None,
                 # DRAM read + write bytes per GEMM launch from one ncu capture of this kernel on the 2-layer case, scaled to
@@ -497,7 +500,9 @@ def main():
             "config": {"workload": res["name"], "l2": "inputs larger than L2 (16 GB of weights streamed every step)",
                        "params": "tau_min 0.1, tau_high 0.85, K_max 8, W_hist 2, sigma2 1.0, k_slow = k_fast = 1, N = L"},
             "tokens_unmasked": tokens, "productive_steps": res["productive"], "gpu_launches": launches, "clocks": res["clocks"],
+            # FLOPs at the burst cuBLAS peak (the stricter bar), and at the rate cuBLAS itself sustains under the power cap
             "step_roofline_ms": step_roof_ms, "step_roofline_frac": step_roof_ms / ms_step,
+            "step_roofline_ms_sustained_peak": step_roof_sus_ms, "step_roofline_frac_sustained_peak": step_roof_sus_ms / ms_step,
             "kernel_ms_per_step": {k: v / res["prof_steps"] for k, v in res["ms_cls"].items()},
             "roofline": roofline, "e2e": res["e2e"]}
     if res["extras"]:
