@@ -2,9 +2,9 @@
 
 Two statements of the same rule live here:
 
-* `slowfast_loop`  — the whole sampling loop written in the shape of Algorithm 1 (outer cycle loop, inner
-  exploratory loop, then the accelerated stage), calling a `predict` callback wherever the algorithm says
-  "Predict r_hat_0 and confidence".  This is the statement a reader checks against the paper.
+* `slowfast_loop`  — the whole sampling loop: cycles of an exploratory stage (`_Sampler.explore`) and an
+  accelerated stage (`_Sampler.accelerate`), each asking a `predict` callback for the greedy tokens and
+  confidences of the rows it reads (Algorithm 1; Section 3.3).
 * `slowfast_step`  — the same rule as a one-step state machine (what a per-step entry point needs); the
   test-suite checks that driving it step by step reproduces `slowfast_loop` exactly.
 
@@ -92,72 +92,84 @@ Predict = Callable[[List[bool], List[int]], Tuple[Dict[int, int], Dict[int, int]
 # predict(masked, rows) -> (a, sq): greedy token and S_q for (at least) the positions in `rows`.
 
 
-def slowfast_loop(L: int, predict: Predict, p: SlowFastParams) -> Tuple[List[Optional[int]], List[StepRecord]]:
-    """Algorithm 1, with the readings R1-R12.  Returns (tokens, trace)."""
-    masked = [True] * L
-    y: List[Optional[int]] = [None] * L
-    k = p.max_steps if p.max_steps > 0 else L           # k <- N
-    s_cycle = 0                                         # s_cycle <- 1 (0-based here)
-    trace: List[StepRecord] = []
+class _Sampler:
+    """Bookkeeping shared by the two stages of a cycle: which positions are still masked, the tokens
+    written so far, the remaining step budget k and the trace."""
 
-    def unmask(positions, a):
-        for i in positions:
-            assert masked[i], "a decoded position was selected again"
-            masked[i] = False
-            y[i] = int(a[i])
+    def __init__(self, L: int, predict: Predict, p: SlowFastParams):
+        self.L, self.predict, self.p = L, predict, p
+        self.masked = [True] * L
+        self.y: List[Optional[int]] = [None] * L
+        self.k = p.max_steps if p.max_steps > 0 else L          # Algorithm 1, initialisation: k = N
+        self.trace: List[StepRecord] = []
 
-    while k > 0 and any(masked):
-        # ---- Phase 1: exploratory stage (slow) ----
-        H: List[int] = []
-        step_count = 0
-        is_stable = False
+    def open_positions(self, lo: int, hi: int) -> List[int]:
+        return [i for i in range(lo, hi) if self.masked[i]]
+
+    def commit(self, phase: int, s: int, hi: int, e_cand: int, stable: bool, chosen: List[int], a: Dict[int, int]):
+        """Writes the greedy tokens of `chosen`, records the step and spends one step of the budget."""
+        for i in chosen:
+            assert self.masked[i], "a decoded position was selected again"
+            self.masked[i] = False
+            self.y[i] = int(a[i])
+        self.trace.append(StepRecord(len(self.trace), phase, s, hi, e_cand, int(stable), chosen, [int(a[i]) for i in chosen]))
+        self.k -= 1
+
+    def last_step(self, phase: int, s: int, hi: int) -> None:
+        """R8: the final permitted step decodes whatever is still masked."""
+        rest = self.open_positions(0, self.L)
+        a, _ = self.predict(list(self.masked), rest)
+        self.commit(phase, s, hi, -1, False, rest, a)
+
+    def explore(self, s: int) -> Optional[int]:
+        """Section 3.3, exploratory stage from window start s.  Returns the span end hi = e_cycle + 1, or None when
+        the sequence (or the budget) ended inside the stage."""
+        p, L = self.p, self.L
+        H: List[int] = []                                         # R5: a fresh history per stage
         e_cand = -1
-        e_cycle = -1
-        while step_count < p.k_max and k > 0 and any(masked):
-            M = [i for i in range(s_cycle, L) if masked[i]]
-            a, sq = predict(list(masked), M)
-            if k == 1:                                  # last permitted step: everything left
-                unmask(M, a)
-                trace.append(StepRecord(len(trace), SLOW, s_cycle, L, -1, 0, M, [int(a[i]) for i in M]))
-                k = 0
-                break
-            above = [i for i in M if exceeds(sq[i], p.tau_min_conf)]
-            e_cand = max(above) if above else min(M)    # end point of convergence
-            chosen = top_k(M, sq, p.k_slow)             # cautious decoding
-            unmask(chosen, a)
+        for _ in range(p.k_max):
+            if self.k == 0 or not any(self.masked):
+                return None
+            if self.k == 1:
+                self.last_step(SLOW, s, L)
+                return None
+            M = self.open_positions(s, L)
+            a, sq = self.predict(list(self.masked), M)
+            reach = [i for i in M if exceeds(sq[i], p.tau_min_conf)]
+            e_cand = reach[-1] if reach else M[0]                 # end point of convergence; R3 when nothing reaches tau_min
             H = (H + [e_cand])[-p.w_hist:]
-            k -= 1
-            step_count += 1
-            if len(H) >= p.w_hist and variance_below(H, p.sigma2_stable):
-                is_stable = True
-                e_cycle = sum(H) // len(H)              # floor of Mean(H_W)
-            trace.append(StepRecord(len(trace), SLOW, s_cycle, L, e_cand, int(is_stable),
-                                    chosen, [int(a[i]) for i in chosen]))
-            if is_stable:
-                break
-        if k == 0 or not any(masked):
-            break
-        if not is_stable:
-            e_cycle = e_cand                            # fallback if no convergence
-        hi = e_cycle + 1
+            stable = len(H) >= p.w_hist and variance_below(H, p.sigma2_stable)
+            self.commit(SLOW, s, L, e_cand, stable, top_k(M, sq, p.k_slow), a)
+            if stable:
+                return sum(H) // len(H) + 1                       # R2: floor of the window's mean
+        return e_cand + 1                                         # K_max steps without stability (Algorithm 1's fallback)
 
-        # ---- Phase 2: accelerated decoding stage (fast) ----
-        while k > 0 and any(masked[s_cycle:hi]):
-            F = [i for i in range(s_cycle, hi) if masked[i]]
-            rest = [i for i in range(L) if masked[i]]
-            a, sq = predict(list(masked), rest if k == 1 else F)
-            if k == 1:
-                unmask(rest, a)
-                trace.append(StepRecord(len(trace), FAST, s_cycle, hi, -1, 0, rest, [int(a[i]) for i in rest]))
-                k = 0
-                break
-            S_high = [i for i in F if exceeds(sq[i], p.tau_high_conf)]
-            chosen = S_high if len(S_high) >= p.min_high_count else top_k(F, sq, p.k_fast)
-            unmask(chosen, a)
-            trace.append(StepRecord(len(trace), FAST, s_cycle, hi, -1, 0, chosen, [int(a[i]) for i in chosen]))
-            k -= 1
-        s_cycle = hi                                    # advance the stable region start
-    return y, trace
+    def accelerate(self, s: int, hi: int) -> None:
+        """Section 3.3, accelerated stage on the span [s, hi); R6: repeated until the span holds no mask."""
+        p = self.p
+        while self.k > 0 and any(self.masked[s:hi]):
+            if self.k == 1:
+                self.last_step(FAST, s, hi)
+                return
+            F = self.open_positions(s, hi)
+            a, sq = self.predict(list(self.masked), F)
+            high = [i for i in F if exceeds(sq[i], p.tau_high_conf)]
+            chosen = high if len(high) >= p.min_high_count else top_k(F, sq, p.k_fast)
+            self.commit(FAST, s, hi, -1, False, chosen, a)
+
+
+def slowfast_loop(L: int, predict: Predict, p: SlowFastParams) -> Tuple[List[Optional[int]], List[StepRecord]]:
+    """The whole sampling loop of Algorithm 1 under the readings R1-R12: cycles of an exploratory stage that
+    locates the span and an accelerated stage that decodes it.  Returns (tokens, trace)."""
+    run = _Sampler(L, predict, p)
+    s_cycle = 0
+    while run.k > 0 and any(run.masked):                          # R7
+        hi = run.explore(s_cycle)
+        if hi is None or run.k == 0 or not any(run.masked):
+            break
+        run.accelerate(s_cycle, hi)
+        s_cycle = hi                                              # the next cycle starts behind the decoded span
+    return run.y, run.trace
 
 
 # ----------------------------------------------------------------------------------------------------
