@@ -197,7 +197,7 @@ int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_t logits_dt
 typedef struct {
     int32_t k_prompt;       /* 100  prompt refresh interval */
     int32_t k_response;     /* 5    response refresh interval */
-    float   rho;            /* 0.25 fraction of the response recomputed on the other steps */
+    double  rho;            /* 0.25 fraction of the response recomputed on the other steps: ceil(rho * gen_len) in double */
 } sfs_cache_params;
 
 /* Switches the cache on for the session (allocating per-layer caches for max_batch x max_seq tokens on the first call)

@@ -11,7 +11,7 @@ response's intermediate features across denoising steps and refreshes them at a 
   In layer l the set R_l of recomputed positions is
         prompt positions, if refresh_p;  plus
         all response positions, if refresh_r;  otherwise the adaptive set: with h = RMSNorm(x) and
-        v_i = h_i Wv^T for the candidate response positions C, the k = min(ceil(rho * L), |C|) candidates (rho as float32) whose
+        v_i = h_i Wv^T for the candidate response positions C, the k = min(ceil(rho * L), |C|) candidates (the product taken in double) whose
         cosine similarity  <v_i, V_l[i]> / (|v_i| |V_l[i]|)  to their cached value is smallest (ties: lower
         position first).  C is every response position in a slow step and the span [s_cycle, hi) in a fast
         step (out-of-span positions keep their cached features while the span is decoded).
@@ -54,8 +54,8 @@ def least_similar(sims: np.ndarray, candidates: Sequence[int], k: int) -> List[i
 
 
 def adaptive_count(rho: float, L: int) -> int:
-    """ceil(rho * L) with rho taken as the float32 the interface carries (as the thresholds of the scheduler are)."""
-    return int(math.ceil(float(np.float32(rho)) * L))
+    """ceil(rho * L), one IEEE double multiply."""
+    return int(math.ceil(float(rho) * float(L)))
 
 
 def cached_forward(cfg: F.ModelConfig, w: Dict, tokens: Sequence[int], P: int, cache: FeatureCache,

@@ -43,7 +43,7 @@ class Params(Structure):
 
 
 class CacheParams(Structure):
-    _fields_ = [("k_prompt", c_int32), ("k_response", c_int32), ("rho", c_float)]
+    _fields_ = [("k_prompt", c_int32), ("k_response", c_int32), ("rho", ctypes.c_double)]
 
 
 STATE_INTS = 32

@@ -238,7 +238,7 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
     s->cache_B = B; s->cache_S = S; s->cache_P = P;
     const sfs_cache_params &cp = s->cache_params;
     const bool rp = (s->cache_t % cp.k_prompt) == 0, rr = (s->cache_t % cp.k_response) == 0;
-    int n_adapt = (int)ceil((double)cp.rho * (double)L);
+    int n_adapt = (int)ceil(cp.rho * (double)L);
     n_adapt = n_adapt < 0 ? 0 : (n_adapt > L ? L : n_adapt);
     const int n_sel = (rp ? P : 0) + (rr ? L : n_adapt);
     if (n_sel_out) *n_sel_out = (rp && rr) ? S : n_sel;
@@ -586,8 +586,8 @@ int32_t sfs_cache_enable(sfs_session *s, const sfs_cache_params *p)
 {
     SFS_REQUIRE(s && s->model, SFS_ERR_INVALID_ARG, "cache_enable: needs a session created from a model");
     if (p == nullptr) { s->cache_on = false; return SFS_OK; }
-    SFS_REQUIRE(p->k_prompt >= 1 && p->k_response >= 1 && p->rho >= 0.f && p->rho <= 1.f, SFS_ERR_INVALID_ARG,
-                "cache_enable: k_prompt %d, k_response %d must be >= 1 and rho %g within [0, 1]", p->k_prompt, p->k_response, (double)p->rho);
+    SFS_REQUIRE(p->k_prompt >= 1 && p->k_response >= 1 && p->rho >= 0.0 && p->rho <= 1.0, SFS_ERR_INVALID_ARG,
+                "cache_enable: k_prompt %d, k_response %d must be >= 1 and rho %g within [0, 1]", p->k_prompt, p->k_response, p->rho);
     const sfs_config &c = s->model->cfg;
     const size_t T = (size_t)s->max_batch * s->max_seq, d = c.d_model;
     if (s->Kc.empty()) {

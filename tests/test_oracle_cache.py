@@ -89,7 +89,9 @@ def test_schedule_counter_and_fast_step_candidates():
         C.cached_forward(CFG, WTS, tt, P, cache, 6, 3, 0.3, span=(3, 6) if step in (1, 4) else None, record=rec)
         seen.append(rec["sets"][0])
     k = C.adaptive_count(0.3, L)
-    assert k == 4 and C.adaptive_count(0.25, 10) == 3 and C.adaptive_count(0.5, 10) == 5      # float32(0.3) * 10 > 3
+    assert k == 3 and C.adaptive_count(0.25, 10) == 3 and C.adaptive_count(0.5, 10) == 5      # ceil(3.0), ceil(2.5), ceil(5.0)
+    assert C.adaptive_count(0.1, 10) == 1 and C.adaptive_count(0.0, 10) == 0 and C.adaptive_count(1.0, 10) == 10
+    assert C.adaptive_count(0.25, 512) == 128 and C.adaptive_count(0.3, 7) == 3
     allr = [P + i for i in range(L)]
     assert seen[0] == list(range(S)) and seen[6] == list(range(S))       # t = 0, 6: both intervals fire
     assert seen[3] == allr                                               # t = 3: response interval only
@@ -116,9 +118,9 @@ def test_least_similar_matches_brute_force_and_picks_the_planted_row():
 def test_changed_token_is_the_least_similar_value_in_the_first_layer():
     t = toks(6)
     cache = C.FeatureCache(CFG, S)
-    C.cached_forward(CFG, WTS, t, P, cache, 100, 100, 0.0625)
+    C.cached_forward(CFG, WTS, t, P, cache, 100, 100, 0.1)
     t2 = t.copy(); t2[P + 7] = 33
     rec = {}
-    C.cached_forward(CFG, WTS, t2, P, cache, 100, 100, 0.0625, record=rec)
-    assert rec["sets"][0] == [P + 7]                                      # k = ceil(0.0625 * 10) = 1 (0.0625 is exact in float32)
+    C.cached_forward(CFG, WTS, t2, P, cache, 100, 100, 0.1, record=rec)
+    assert rec["sets"][0] == [P + 7]                                      # k = ceil(0.1 * 10) = 1
     assert np.allclose(np.delete(rec["sims"][0], 7), 1.0)                 # layer 0 sees only the embeddings
