@@ -215,6 +215,13 @@ int32_t sfs_forward_cached(sfs_session *session, const int32_t *d_tokens, int32_
                            const sfs_state *d_state, const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
                            void *d_logits, int32_t logits_dtype, int32_t *d_sets, float *d_sims, int32_t *n_sel, void *stream);
 
+/* Inspection of cached generation: from now on every cached step that sfs_generate_steps enqueues also writes its
+ * recomputed token indices to d_sets [n_layers, B, n_sel] and, on adaptive steps, the similarities to d_sims
+ * [n_layers, B, gen_len], exactly as sfs_forward_cached does (n_sel follows from the step counter: S on a step that
+ * refreshes prompt and response, else (P if the prompt is refreshed) + (gen_len if the response is, else
+ * ceil(rho * gen_len))).  The buffers are overwritten by every step; NULL pointers switch the dumps off. */
+int32_t sfs_cache_dump(sfs_session *session, int32_t *d_sets, float *d_sims);
+
 /* ---- the whole loop ------------------------------------------------------------------------------------ */
 
 /* Algorithm 1 for B independent sequences with a common prompt length P and response length gen_len:

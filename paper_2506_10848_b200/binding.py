@@ -199,6 +199,10 @@ def sfs_cache_reset(session):
     _check(lib().sfs_cache_reset(session))
 
 
+def sfs_cache_dump(session, sets=None, sims=None):
+    _check(lib().sfs_cache_dump(session, _ptr(sets), _ptr(sims)))
+
+
 def sfs_forward_cached(session, tokens, B, S, P, state, rows, n_rows_dev, max_rows, logits, logits_dtype, sets=None, sims=None,
                        stream=None):
     """Returns n_sel, the number of recomputed rows per sequence and layer in this step."""

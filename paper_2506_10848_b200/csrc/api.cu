@@ -619,6 +619,13 @@ int32_t sfs_cache_reset(sfs_session *s)
     return SFS_OK;
 }
 
+int32_t sfs_cache_dump(sfs_session *s, int32_t *d_sets, float *d_sims)
+{
+    SFS_REQUIRE(s && s->model, SFS_ERR_INVALID_ARG, "cache_dump: needs a session created from a model");
+    s->dump_sets = d_sets; s->dump_sims = d_sims;
+    return SFS_OK;
+}
+
 int32_t sfs_forward_cached(sfs_session *s, const int32_t *d_tokens, int32_t B, int32_t S, int32_t P,
                            const sfs_state *d_state, const int32_t *d_rows, const int32_t *d_n_rows, int32_t max_rows,
                            void *d_logits, int32_t logits_dtype, int32_t *d_sets, float *d_sims, int32_t *n_sel, void *stream)
@@ -693,7 +700,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         const int cur = s->gen_cur, nxt = cur ^ 1;
         const int32_t *d_active = s->ctrl + 2;
         const int32_t *rows = s->rows[cur], *n_rows = s->ctrl + cur;
-        if (s->cache_on) rc = run_body_cached(s, s->tokens, B, S, P, s->state, d_active, nullptr, nullptr, nullptr, st);
+        if (s->cache_on) rc = run_body_cached(s, s->tokens, B, S, P, s->state, d_active, s->dump_sets, s->dump_sims, nullptr, st);
         else rc = run_body(s, s->tokens, B, S, d_active, st);
         if (rc != SFS_OK) return rc;
         if ((rc = timed_launch(s, SFS_K_RMSNORM, st, [&] { return launch_rmsnorm(s->x, s->pending_ptr, s->pending_n, s->pending_stride, s->model->final_norm, s->hfin, rows, n_rows, B * L, c.d_model, c.rms_eps, st); })) != SFS_OK) return rc;

@@ -64,6 +64,7 @@ struct sfs_session {
     __nv_bfloat16 *vnew_t = nullptr;         // [d, T] fresh values of every row, transposed
     float *sim_partial = nullptr;            // [kSimSlices, T, 3]
     int32_t *sel_rows = nullptr;             // [T] rows recomputed in the current layer
+    int32_t *dump_sets = nullptr; float *dump_sims = nullptr;   // caller's buffers for the sets / similarities of generate steps
     std::vector<CacheLayerPlans> cache_plans;
     std::map<int, std::vector<GatherLayerPlans>> gather_plans;
     // generation bookkeeping (host)

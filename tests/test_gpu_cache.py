@@ -138,3 +138,103 @@ def test_generation_with_cache_finishes_and_decodes_every_position_once():
     assert np.all(n_sel.sum(axis=0) == L)                                # every position unmasked exactly once
     sfs.sfs_session_destroy(session)
     model.close()
+
+
+def replay_cached_generation(shape, model, cfg, w_or, B, P, L, kp, kr, rho, max_steps, logits_ok, cache_dtype=np.float64, seed=0):
+    """Teacher-forced cached generation: the device loop runs with the cache on, one step at a time, dumping its logits, row
+    list and per-layer recomputed sets.  Per step and sequence the oracle's cached forward pass is run on the oracle's own
+    token state under the sets the GPU chose (logits within tolerance; the sets themselves must be the oracle's rule applied
+    to the GPU's similarities), then the oracle's row statistics and scheduler, fed the GPU's logits, must reproduce the
+    GPU's decisions and tokens exactly.  Returns the number of steps replayed and the tokens unmasked per sequence."""
+    from oracle import rowstats as RS
+    from oracle.scheduler import FAST, SlowFastParams, SlowFastState, rows_needed, slowfast_step
+    S, nl = P + L, shape.n_layers
+    po = SlowFastParams()
+    pg = sfs.Params.default()
+    prompt = W.prompt_ids(B, P, shape.vocab - 2, seed=seed)
+    n_adapt = C.adaptive_count(rho, L)
+    session = sfs.sfs_session_create(model, B, S)
+    try:
+        sfs.sfs_cache_enable(session, kp, kr, rho)
+        trace = torch.zeros((max_steps, B, sfs.TRACE_INTS), dtype=torch.int32, device=DEV)
+        dump = torch.zeros((B * L, shape.vocab), dtype=torch.bfloat16, device=DEV)
+        rows_d = torch.zeros(B * L, dtype=torch.int32, device=DEV)
+        nrows_d = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sets = torch.full((nl * B * S,), -1, dtype=torch.int32, device=DEV)
+        sims = torch.zeros((nl * B * L,), dtype=torch.float32, device=DEV)
+        sfs.sfs_cache_dump(session, sets, sims)
+        sfs.sfs_generate_begin(session, prompt.to(DEV), B, P, L, pg)
+        st = [SlowFastState.fresh(L, po) for _ in range(B)]
+        tok = [prompt[b].tolist() + [shape.mask_id] * L for b in range(B)]
+        caches = [C.FeatureCache(cfg, S, dtype=cache_dtype) for _ in range(B)]
+        n_unmasked = [0] * B
+        step = 0
+        while step < max_steps and not all(s_.done for s_ in st):
+            sets.fill_(-1)
+            sfs.sfs_generate_steps(session, 1, trace, max_steps, dump, rows_d, nrows_d)
+            torch.cuda.synchronize()
+            rp, rr = step % kp == 0, step % kr == 0
+            n_sel = S if (rp and rr) else (P if rp else 0) + (L if rr else n_adapt)
+            gsets = sets.cpu().numpy()[: nl * B * n_sel].reshape(nl, B, n_sel)
+            gsims = sims.cpu().numpy().reshape(nl, B, L)
+            need = [(b, i) for b in range(B) for i in rows_needed(st[b])]
+            n = int(nrows_d.item())
+            assert rows_d[:n].tolist() == [b * S + P + i for (b, i) in need], step
+            lg = dump[:n].cpu()
+            got = lg.float().numpy().astype(np.float64)
+            stats = RS.row_stats(W.bf16_bits(lg))
+            for b in range(B):
+                if st[b].done:
+                    continue
+                fast = st[b].phase == FAST
+                span = (st[b].s_cycle, st[b].hi) if fast else None
+                forced = lambda l, s_, c_, b=b: sorted(set(int(r) - b * S - P for r in gsets[l][b] if int(r) - b * S >= P))
+                rec_c = {}
+                idx = {i: j for j, (bb, i) in enumerate(need) if bb == b}
+                mine = sorted(idx)
+                ref = C.cached_forward(cfg, w_or, np.asarray(tok[b]), P, caches[b], kp, kr, rho, span=span, rows=[P + i for i in mine],
+                                       select=forced, record=rec_c).astype(np.float64)
+                logits_ok(step, b, got[[idx[i] for i in mine]], ref)
+                for l in range(nl):
+                    assert sorted(set(int(r) - b * S for r in gsets[l][b])) == rec_c["sets"][l], (step, b, l)
+                    if not rr and n_adapt > 0:
+                        cand = list(range(L)) if not fast else list(range(span[0], span[1]))
+                        assert forced(l, None, None) == C.least_similar(gsims[l][b][cand], cand, min(n_adapt, len(cand))), (step, b, l)
+                rec = slowfast_step(st[b], {i: int(stats["argmax"][j]) for i, j in idx.items()}, {i: int(stats["sq"][j]) for i, j in idx.items()}, po)
+                for i, t in zip(rec.positions, rec.tokens):
+                    tok[b][P + i] = t
+                n_unmasked[b] += len(rec.positions)
+                assert trace[step, b].tolist()[:6] == [rec.phase, rec.s, rec.hi, rec.e_cand, rec.stable, len(rec.positions)], (step, b, rec)
+            step += 1
+        out = torch.zeros((B, S), dtype=torch.int32, device=DEV)
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+        sfs.sfs_generate_end(session, out, state)
+        sfs.sfs_check_device_status()
+        o = out.cpu().tolist()
+        for b in range(B):
+            assert o[b] == tok[b], b                       # tokens written so far, masked positions still hold the mask id
+            assert int(state[b, sfs.STATE_FIELDS.index("n_masked")]) == L - n_unmasked[b]
+        return step, n_unmasked
+    finally:
+        sfs.sfs_cache_dump(session, None, None)
+        sfs.sfs_cache_enable(session, 1, 1, 0.0, off=True)
+        sfs.sfs_session_destroy(session)
+
+
+@pytest.mark.parametrize("B,kp,kr,rho", [(2, 100, 4, 0.25), (1, 6, 3, 0.5)])
+def test_cached_generation_is_reproduced_by_the_oracle_step_by_step(B, kp, kr, rho):
+    """The whole cached decode loop on the tiny model (logit scale 60: slow and fast steps, spans, parallel unmasking)."""
+    shape, model, cfg, w64 = tiny_setup(seed=0, logit_scale=60.0)
+    P, L = 32, 64
+
+    def logits_ok(step, b, got, ref):
+        err = np.abs(got - ref)
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        assert rel <= REL_L2, (step, b, rel)
+        assert np.all(err <= max_abs_bar(shape.logit_scale) + 2.0 ** -8 * np.abs(ref)), (step, b, err.max())   # + rounding of the stored bf16 logit
+
+    try:
+        steps, n_unmasked = replay_cached_generation(shape, model, cfg, w64, B, P, L, kp, kr, rho, L, logits_ok)
+        assert n_unmasked == [L] * B and steps < L                 # finished, with parallel unmasking on the way
+    finally:
+        model.close()
