@@ -122,7 +122,9 @@ int32_t sfs_session_destroy(sfs_session *session);
 /* ---- the steps of one denoising iteration ----------------------------------------------------------- */
 
 /* Eq. 2: logits of the mask predictor for the listed rows.
- *   d_tokens [B, S] int32 (masked positions must hold mask_id); d_rows [>= n_rows] flat token indices, or
+ *   d_tokens [B, S] int32.  There is no separate mask argument: the predictor's input IS the token sequence, in which
+ *   a masked position holds the [MASK] token's id (Section 3.1: y^(k) is a sequence over the vocabulary that contains
+ *   [MASK]); which positions are masked matters only to sfs_select, which takes the mask array.  d_rows [>= n_rows] flat token indices, or
  *   NULL for all B*S rows in order; n_rows is read from the device scalar d_n_rows when it is not NULL
  *   (then max_rows bounds it and sizes the launch), else it is max_rows.
  *   d_logits [max_rows, vocab] row-major, bf16 or fp32 per logits_dtype; row r belongs to d_rows[r]. */
@@ -153,7 +155,8 @@ int32_t sfs_state_init(sfs_state *d_state, int32_t B, int32_t gen_len, const sfs
  *   d_logits [n_rows, ld]; d_rows [n_rows] flat token indices b*S + pos the logits rows belong to; a
  *   sequence's step needs the rows of its masked positions in [s_cycle, L) (slow), [s_cycle, hi) (fast) or
  *   all of them (k_remaining == 1); extra rows are ignored, a missing one sets state.status =
- *   SFS_ERR_MISSING_ROW and leaves the sequence untouched.
+ *   SFS_ERR_MISSING_ROW and leaves the sequence untouched.  A row index outside [0, B*S) is skipped (nothing is
+ *   written for it) and reported as SFS_ERR_INVALID_ARG by sfs_check_device_status.
  *   Outputs: d_sel_count [B], d_sel_pos / d_sel_tok [B, L] (response positions ascending, and their tokens);
  *   optional d_next_rows [B*L] + d_next_n_rows [1]: the rows the following step will need, sequence-major;
  *   optional d_trace [B, SFS_TRACE_INTS]: (phase, s_cycle, hi, e_cand, stable, n_sel, n_masked_after,
@@ -174,7 +177,9 @@ int32_t sfs_select(sfs_session *session, const void *d_logits, int32_t logits_dt
  *   by every GPU that loads the library until the process exits.  The call itself performs no cudaMalloc / cudaFree
  *   and calls no allocating routine.  All calls share the array: it keeps the previous call's contents (the call
  *   clears the parts that must start at zero), and calls whose kernels may overlap on the GPU race - run them one
- *   after another.  The first call on each device looks up the array's address; make it before any stream capture. */
+ *   after another.  The first call on each device looks up the array's address; make it before any stream capture.
+ *   Device-side conditions of the call (a row index outside [0, B*S), a bounded wait that gave up) are written to
+ *   d_state[b].status of the call's sequences, since this entry has no session or status word to report them through. */
 #define SFS_STATIC_MAX_POSITIONS 16384
 #define SFS_STATIC_MAX_BATCH 64
 int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_t logits_dtype, int64_t ld,

@@ -36,18 +36,18 @@ static int32_t check_params(const sfs_params *p)
     return SFS_OK;
 }
 
-// one sticky device status word per process (set by kernels whose bounded waits give up)
-static int32_t *g_status_word = nullptr;
+// one sticky status word per device
+static int32_t *g_status_word[kMaxDevices] = {};
 int32_t *device_status_word()
 {
-    if (!g_status_word) {
-        if (cudaMalloc(&g_status_word, 256) != cudaSuccess) { g_status_word = nullptr; return nullptr; }
-        cudaMemset(g_status_word, 0, 256);
+    int32_t *&w = g_status_word[current_device_slot()];
+    if (!w) {
+        if (cudaMalloc(&w, 256) != cudaSuccess) { w = nullptr; return nullptr; }
+        cudaMemset(w, 0, 256);
     }
-    return g_status_word;
+    return w;
 }
-// the word if some earlier call has created it, else null: never allocates
-int32_t *device_status_word_if_any() { return g_status_word; }
+int32_t *device_status_word_if_any() { return g_status_word[current_device_slot()]; }
 
 template <typename T>
 static int32_t dev_alloc(sfs_session *s, T **out, size_t count, bool zero)
@@ -452,6 +452,7 @@ int32_t sfs_select_session_create(int32_t vocab, int32_t max_batch, int32_t max_
     s->max_batch = max_batch; s->max_seq = max_seq; s->vocab = vocab;
     int32_t rc = session_alloc_select(s);
     if (rc != SFS_OK) { sfs_session_destroy(s); return rc; }
+    if (device_status_word() == nullptr) { sfs_session_destroy(s); set_error("cannot allocate the device status word"); return SFS_ERR_OOM; }
     SFS_CUDA(cudaDeviceSynchronize());
     *out = s;
     return SFS_OK;
@@ -537,7 +538,8 @@ int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab,
     SFS_REQUIRE(max_rows >= 0, SFS_ERR_INVALID_ARG, "max_rows %d", max_rows);
     SFS_REQUIRE(aligned_to(d_logits, logits_dtype == SFS_LOGITS_BF16 ? 2 : 4), SFS_ERR_INVALID_ARG, "d_logits misaligned");
     return launch_row_stats(d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, nullptr, d_argmax,
-                            reinterpret_cast<unsigned long long *>(d_sq), d_conf, nullptr, nullptr, (cudaStream_t)stream);
+                            reinterpret_cast<unsigned long long *>(d_sq), d_conf, nullptr, nullptr, 0, device_status_word_if_any(),
+                            (cudaStream_t)stream);
 }
 
 int32_t sfs_state_init(sfs_state *d_state, int32_t B, int32_t gen_len, const sfs_params *params, void *stream)
@@ -568,7 +570,7 @@ int32_t sfs_select(sfs_session *s, const void *d_logits, int32_t logits_dtype, i
     if (rc != SFS_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     rc = launch_row_stats(d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, d_rows, nullptr, nullptr, nullptr,
-                          s->pos_sq, s->pos_arg, st);
+                          s->pos_sq, s->pos_arg, B * S, device_status_word(), st);
     if (rc != SFS_OK) return rc;
     SelectArgs a{};
     a.tokens = d_tokens; a.mask = d_mask; a.B = B; a.S = S; a.P = P; a.L = S - P;
@@ -712,7 +714,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         }
         if ((rc = timed_launch(s, SFS_K_ROW_STATS, st, [&] {
                  return launch_row_stats(s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, nullptr, nullptr, nullptr,
-                                         s->pos_sq, s->pos_arg, st); })) != SFS_OK) return rc;
+                                         s->pos_sq, s->pos_arg, B * S, err, st); })) != SFS_OK) return rc;
         SelectArgs a{};
         a.tokens = s->tokens; a.mask = s->mask; a.B = B; a.S = S; a.P = P; a.L = L;
         a.state = s->state; a.params = s->gen_params;

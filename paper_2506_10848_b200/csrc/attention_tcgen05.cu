@@ -294,10 +294,11 @@ int32_t launch_dh(const AttnPlan &p, int kq, const int32_t *d_active, int32_t *e
 {
     constexpr size_t smem = (size_t)QT * DH * 2 + KV_STAGES * (size_t)(KT * DH * 2 + DH * KT * 2) + QT * KT * 2
                           + kAttnBars * 8 + 16 + 1024;
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};
+    bool &done = configured[current_device_slot()];
+    if (!done) {
         SFS_CUDA(cudaFuncSetAttribute(attention_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured = true;
+        done = true;
     }
     AttnArgs a = p.args;
     a.err = err; a.d_active = d_active;

@@ -555,10 +555,11 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
 {
     // always ask for more than half of an SM's shared memory: one CTA per SM, so the allocation of all 512
     // tensor-memory columns can never wait for a co-resident CTA
-    static bool configured = false;
-    if (!configured) {
+    static bool configured[kMaxDevices] = {};
+    bool &done = configured[current_device_slot()];
+    if (!done) {
         SFS_CUDA(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
-        configured = true;
+        done = true;
     }
     GemmArgs g = p.args;
     g.d_m = d_m; g.err = err; g.d_active = d_active;

@@ -16,7 +16,6 @@
 namespace cg = cooperative_groups;
 
 namespace sfs {
-int32_t *device_status_word_if_any();     // the process's sticky status word, null until some call has created it
 namespace {
 
 constexpr float kLog2e = 0x1.715476p+0f;
@@ -100,6 +99,8 @@ struct RowOut {
     const int32_t *rows;            // flat token index per logits row, or null
     int32_t *argmax; unsigned long long *sq; float *conf;       // dense by logits row (optional)
     unsigned long long *pos_sq; int32_t *pos_arg;               // scattered by flat token index (optional)
+    int32_t n_positions;                                        // size of the scattered arrays
+    int32_t *err;                                               // device status word (optional)
 };
 
 __device__ __forceinline__ void write_row(const RowOut &o, int row, int arg, unsigned long long S) {
@@ -108,8 +109,12 @@ __device__ __forceinline__ void write_row(const RowOut &o, int row, int arg, uns
     if (o.conf) o.conf[row] = (float)((double)(1u << SFS_CONF_QBITS) / (double)S);
     if (o.rows && o.pos_sq) {
         const int p = o.rows[row];
-        o.pos_sq[p] = S;
-        o.pos_arg[p] = arg;
+        if ((unsigned)p < (unsigned)o.n_positions) {
+            o.pos_sq[p] = S;
+            o.pos_arg[p] = arg;
+        } else if (o.err) {
+            atomicExch(o.err, SFS_ERR_INVALID_ARG);               // a row index outside the token grid: skipped, reported
+        }
     }
 }
 
@@ -376,8 +381,7 @@ int32_t launch_staged(const uint4 *logits, long long ld_chunks, int nchunks, int
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)kStagedCluster; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_staged_bf16, logits, ld_chunks, nchunks, per_cta, vocab, d_n_rows, max_rows, out,
-                                device_status_word_if_any()));
+    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_staged_bf16, logits, ld_chunks, nchunks, per_cta, vocab, d_n_rows, max_rows, out, out.err));
     return SFS_OK;
 }
 
@@ -447,8 +451,7 @@ int32_t launch_cluster(const uint4 *logits, long long ld_chunks, int nchunks, in
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)C; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_cluster_bf16<NV>, logits, ld_chunks, nchunks, vocab, d_n_rows, max_rows, out,
-                                device_status_word_if_any()));
+    SFS_CUDA(cudaLaunchKernelEx(&cfg, rowstats_cluster_bf16<NV>, logits, ld_chunks, nchunks, vocab, d_n_rows, max_rows, out, out.err));
     return SFS_OK;
 }
 
@@ -457,10 +460,11 @@ int32_t launch_cluster(const uint4 *logits, long long ld_chunks, int nchunks, in
 int32_t launch_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
                          const int32_t *d_n_rows, int32_t max_rows, const int32_t *d_rows,
                          int32_t *d_argmax, unsigned long long *d_sq, float *d_conf,
-                         unsigned long long *d_pos_sq, int32_t *d_pos_arg, cudaStream_t stream)
+                         unsigned long long *d_pos_sq, int32_t *d_pos_arg, int32_t n_positions, int32_t *d_err,
+                         cudaStream_t stream)
 {
     if (max_rows <= 0) return SFS_OK;
-    RowOut out{d_rows, d_argmax, d_sq, d_conf, d_pos_sq, d_pos_arg};
+    RowOut out{d_rows, d_argmax, d_sq, d_conf, d_pos_sq, d_pos_arg, n_positions, d_err};
     const bool fast = logits_dtype == SFS_LOGITS_BF16 && (vocab % 8) == 0 && (ld % 8) == 0 && aligned_to(d_logits, 16);
     if (fast) {
         const int nchunks = vocab / 8;

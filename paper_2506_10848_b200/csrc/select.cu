@@ -181,7 +181,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
         // the statistics of this step are consumed: a later step must bring its own
         for (int i = tid; i < L; i += kSelThreads) psq[i] = 0;
     } else {
-        for (int i = tid; i < L; i += kSelThreads) s_sel[i] = 0;
+        // a finished (or stopped) sequence consumes the statistics supplied for it as well: nothing stale is left for a
+        // later generation that reuses the scratch
+        for (int i = tid; i < L; i += kSelThreads) { s_sel[i] = 0; psq[i] = 0; }
     }
     __syncthreads();
 

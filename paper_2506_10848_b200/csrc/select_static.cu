@@ -24,20 +24,30 @@ struct StaticScratch {
     int32_t seq_rows[SFS_STATIC_MAX_POSITIONS];
     int32_t seq_row_count[SFS_STATIC_MAX_BATCH];
     int32_t ticket[4];
+    int32_t status[4];            // [0]: device status of the call in flight (a bounded wait that gave up, a row index outside the grid)
 };
 
 // In host code this name is only a handle for the runtime, not a device address: it is never passed to a kernel.
 static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
 
-constexpr int kMaxDevices = 64;
-StaticScratch *g_scratch_ptr[kMaxDevices] = {};
+StaticScratch *g_scratch_ptr[sfs::kMaxDevices] = {};
+
+// folds the call's device status into every sequence's state.status (first error wins), so that a caller that may not
+// allocate still sees a device-side failure where it already looks
+__global__ void fold_status_kernel(const int32_t *status, sfs_state *state, int B)
+{
+    const int32_t s = *status;
+    if (s == SFS_OK) return;
+    for (int b = threadIdx.x; b < B; b += blockDim.x)
+        if (state[b].status == SFS_OK) state[b].status = s;
+}
 
 // device address of the array on the current device, looked up once per device
 int32_t scratch_for_current_device(StaticScratch **out)
 {
     int dev = -1;
     SFS_CUDA(cudaGetDevice(&dev));
-    SFS_REQUIRE(dev >= 0 && dev < kMaxDevices, SFS_ERR_UNSUPPORTED, "device ordinal %d not supported", dev);
+    SFS_REQUIRE(dev >= 0 && dev < sfs::kMaxDevices, SFS_ERR_UNSUPPORTED, "device ordinal %d not supported", dev);
     if (g_scratch_ptr[dev] == nullptr) {
         void *p = nullptr;
         SFS_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
@@ -76,9 +86,9 @@ extern "C" int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_
     cudaStream_t st = (cudaStream_t)stream;
     // the array keeps what the previous call left: everything that must start at zero is cleared here
     SFS_CUDA(cudaMemsetAsync(sc->pos_sq, 0, sizeof(unsigned long long) * (size_t)B * S, st));
-    SFS_CUDA(cudaMemsetAsync(sc->ticket, 0, sizeof(sc->ticket), st));
+    SFS_CUDA(cudaMemsetAsync(sc->ticket, 0, sizeof(sc->ticket) + sizeof(sc->status), st));
     rc = launch_row_stats(d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, d_rows, nullptr, nullptr, nullptr,
-                          sc->pos_sq, sc->pos_arg, st);
+                          sc->pos_sq, sc->pos_arg, B * S, sc->status, st);
     if (rc != SFS_OK) return rc;
     SelectArgs a{};
     a.tokens = d_tokens; a.mask = d_mask; a.B = B; a.S = S; a.P = P; a.L = S - P;
@@ -88,5 +98,8 @@ extern "C" int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_
     a.seq_rows = sc->seq_rows; a.seq_row_count = sc->seq_row_count;
     a.next_rows = d_next_rows; a.next_n_rows = d_next_n_rows; a.n_active = nullptr;
     a.ticket = sc->ticket; a.trace = d_trace;
-    return launch_select(a, st);
+    if ((rc = launch_select(a, st)) != SFS_OK) return rc;
+    fold_status_kernel<<<1, 64, 0, st>>>(sc->status, d_state, B);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
 }

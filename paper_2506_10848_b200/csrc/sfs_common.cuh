@@ -34,6 +34,19 @@ void set_error(const char *fmt, ...);          // stores a message for sfs_last_
 
 static inline bool aligned_to(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// Per-device bookkeeping (kernel attributes, the sticky status word) is indexed by the ordinal of the current device.
+constexpr int kMaxDevices = 64;
+static inline int current_device_slot()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    return dev;
+}
+// The current device's sticky status word (set by kernels whose bounded waits give up, or that skip an invalid row);
+// allocated on first use, null if that allocation fails.  The _if_any form never allocates.
+int32_t *device_status_word();
+int32_t *device_status_word_if_any();
+
 // ---- device helpers ---------------------------------------------------------------------------------
 #ifdef __CUDACC__
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h16) { return __uint_as_float(h16 << 16); }
@@ -73,11 +86,13 @@ __device__ __forceinline__ int warp_max_i32(int v) {
 // ---- internal launchers (defined in the .cu files) --------------------------------------------------
 // Row statistics (Section 3.1: greedy token and confidence).  Results are written densely by logits row
 // (d_argmax/d_sq/d_conf, each optional) and, when d_rows is given, scattered to d_pos_sq/d_pos_arg at the
-// flat token index of each row.
+// flat token index of each row; an index outside [0, n_positions) is skipped and reported as SFS_ERR_INVALID_ARG
+// in *d_err (a device status word, optional), as is a bounded wait that gives up (SFS_ERR_TIMEOUT).
 int32_t launch_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
                          const int32_t *d_n_rows, int32_t max_rows, const int32_t *d_rows,
                          int32_t *d_argmax, unsigned long long *d_sq, float *d_conf,
-                         unsigned long long *d_pos_sq, int32_t *d_pos_arg, cudaStream_t stream);
+                         unsigned long long *d_pos_sq, int32_t *d_pos_arg, int32_t n_positions, int32_t *d_err,
+                         cudaStream_t stream);
 
 struct SelectArgs {
     int32_t *tokens; uint8_t *mask; int32_t B, S, P, L;

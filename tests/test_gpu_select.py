@@ -180,3 +180,64 @@ def test_epilogue_microbenchmark_one_slow_one_fast_step():
                 assert n > 1                               # several in-span rows exceed tau_high: parallel unmasking
     finally:
         sfs.sfs_session_destroy(session)
+
+
+def _one_step_inputs(B, P, L, V, pg, gen):
+    S = P + L
+    tokens = torch.full((B, S), V - 1, dtype=torch.int32, device=DEV)
+    mask = torch.zeros((B, S), dtype=torch.uint8, device=DEV); mask[:, P:] = 1
+    state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+    sfs.sfs_state_init(state, B, L, pg)
+    rows = torch.tensor([b * S + P + i for b in range(B) for i in range(L)], dtype=torch.int32, device=DEV)
+    logits = synthetic_step_logits(B * L, V, gen, torch.bfloat16).to(DEV)
+    return tokens, mask, state, rows, logits
+
+
+def test_row_index_outside_the_token_grid_is_skipped_and_reported():
+    """A row list may carry a stale or foreign index: the statistics of such a row are dropped (never written outside the
+    scratch), the device status word reports it, and the sequence whose row is now missing stops with MISSING_ROW."""
+    B, P, L, V = 2, 4, 24, 512
+    S = P + L
+    po, pg = params_pair()
+    session = sfs.sfs_select_session_create(V, B, S)
+    try:
+        tokens, mask, state, rows, logits = _one_step_inputs(B, P, L, V, pg, torch.Generator().manual_seed(5))
+        bad = rows.clone()
+        bad[3] = B * S + 1000                               # sequence 0's row 3: beyond the grid
+        bad[L + 7] = -9                                     # sequence 1's row 7: negative
+        before = tokens.clone()
+        sfs.sfs_select(session, logits, sfs.LOGITS_BF16, V, bad, None, B * L, tokens, mask, B, S, P, state, pg)
+        with pytest.raises(sfs.SfsError) as e:
+            sfs.sfs_check_device_status()
+        assert e.value.status == sfs.ERR_INVALID_ARG
+        sfs.sfs_check_device_status()                       # sticky word is cleared by the read
+        for b in range(B):
+            assert state_to_dict(state[b])["status"] == sfs.ERR_MISSING_ROW
+        assert torch.equal(tokens, before) and int(mask[:, P:].sum()) == B * L
+    finally:
+        sfs.sfs_session_destroy(session)
+
+
+def test_statistics_of_a_finished_sequence_do_not_survive_into_the_next_generation():
+    """Rows supplied for a sequence that is already done are consumed like any others: when the scratch is reused with a
+    fresh state, a needed row that the caller omits is reported as missing instead of being read from the old call."""
+    B, P, L, V = 1, 0, 16, 512
+    S = P + L
+    po, pg = params_pair(max_steps=1)                       # one permitted step: it decodes everything, the sequence is done
+    gen = torch.Generator().manual_seed(6)
+    session = sfs.sfs_select_session_create(V, B, S)
+    try:
+        tokens, mask, state, rows, logits = _one_step_inputs(B, P, L, V, pg, gen)
+        sfs.sfs_select(session, logits, sfs.LOGITS_BF16, V, rows, None, L, tokens, mask, B, S, P, state, pg)
+        assert state_to_dict(state[0])["done"] == 1
+        # statistics for the finished sequence arrive once more (a caller running a batch does this for finished members)
+        sfs.sfs_select(session, logits, sfs.LOGITS_BF16, V, rows, None, L, tokens, mask, B, S, P, state, pg)
+        # new generation on the same scratch; row 5 is left out
+        _, pg2 = params_pair()
+        tokens, mask, state, rows, logits = _one_step_inputs(B, P, L, V, pg2, gen)
+        keep = [i for i in range(L) if i != 5]
+        sfs.sfs_select(session, logits[keep].contiguous(), sfs.LOGITS_BF16, V, rows[keep].contiguous(), None, L - 1, tokens, mask, B, S, P, state, pg2)
+        sfs.sfs_check_device_status()
+        assert state_to_dict(state[0])["status"] == sfs.ERR_MISSING_ROW and int(mask.sum()) == L
+    finally:
+        sfs.sfs_session_destroy(session)

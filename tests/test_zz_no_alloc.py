@@ -43,9 +43,13 @@ def test_static_entry_matches_session_entry_on_consecutive_calls():
             n_dev = torch.tensor([n_rows], dtype=torch.int32, device=DEV)
             sfs.sfs_select(session, logits, sfs.LOGITS_BF16, V, rows, n_dev, n_rows, a["tokens"], a["mask"], B, S, P, a["state"], pg,
                            a["sel_count"], a["sel_pos"], a["sel_tok"], a["next_rows"], a["next_n"], a["trace"])
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             sfs.sfs_select_static(V, logits, sfs.LOGITS_BF16, V, rows, n_dev, n_rows, b["tokens"], b["mask"], B, S, P, b["state"], pg,
                                   b["sel_count"], b["sel_pos"], b["sel_tok"], b["next_rows"], b["next_n"], b["trace"])
             torch.cuda.synchronize()
+            if call > 0:                                    # (the very first call may load the kernels' code)
+                assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the amount of free device memory"
             for key in ("tokens", "mask", "state", "sel_count", "next_n", "trace"):
                 assert torch.equal(a[key], b[key]), (call, key)
             for q in range(B):
@@ -70,3 +74,18 @@ def test_static_entry_rejects_sizes_beyond_its_array():
     with pytest.raises(sfs.SfsError) as e:
         sfs.sfs_select_static(64, t, sfs.LOGITS_BF16, 64, t, None, 1, t, t, sfs.STATIC_MAX_BATCH + 1, 8, 0, t, pg)
     assert e.value.status == sfs.ERR_UNSUPPORTED
+
+
+def test_static_entry_reports_a_bad_row_index_in_the_sequence_state():
+    """No session, hence no process-wide status word to read: a row index outside the token grid is skipped (nothing is
+    written outside the built-in array) and shows up as state.status of the sequences of that call."""
+    B, P, L, V = 1, 0, 16, 256
+    pg = sfs.Params.default()
+    d = fresh(B, P, L, V, pg)
+    rows = torch.arange(L, dtype=torch.int32, device=DEV)
+    rows[2] = sfs.STATIC_MAX_POSITIONS * 64                # far outside
+    logits = (torch.randn((L, V), generator=torch.Generator().manual_seed(1)) * 2).to(torch.bfloat16).to(DEV)
+    sfs.sfs_select_static(V, logits, sfs.LOGITS_BF16, V, rows, None, L, d["tokens"], d["mask"], B, L, P, d["state"], pg)
+    torch.cuda.synchronize()
+    status = int(d["state"][0, sfs.STATE_FIELDS.index("status")])
+    assert status in (sfs.ERR_MISSING_ROW, sfs.ERR_INVALID_ARG) and int(d["mask"].sum()) == L
