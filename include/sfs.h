@@ -48,6 +48,10 @@ extern "C" {
 #define SFS_PHASE_SLOW 0           /* exploratory stage (Section 3.3, stage 1) */
 #define SFS_PHASE_FAST 1           /* accelerated decoding stage (Section 3.3, stage 2) */
 
+#define SFS_SAMPLER_SLOWFAST       0
+#define SFS_SAMPLER_LOW_CONFIDENCE 1
+#define SFS_SAMPLER_RANDOM         2
+
 #define SFS_CONF_QBITS 28          /* S_q = sum_v trunc(2^28 * exp(x_v - max x)) */
 #define SFS_MAX_W_HIST 8
 #define SFS_TRACE_INTS 8
@@ -85,6 +89,21 @@ typedef struct {
     int32_t k_fast;           /* 1     tokens unmasked by the fallback of an accelerated step */
     int32_t max_steps;        /* N; 0 means N = gen_len */
     int32_t min_high_count;   /* 1     fallback when fewer positions than this exceed tau_high_conf */
+    /* The transition rule S of Eq. 4.  0 is the SlowFast rule; 1 and 2 are the LLaDA strategies of Section 3.1 that the
+     * paper's tables use as the 1.00x baseline, on the same engine.  With N = max_steps (0: N = gen_len) and k = N .. 1:
+     *   1 low-confidence remasking: after step k, floor(L_b * (1 - (k_b - 1) / N_b)) positions of the current block are
+     *     unmasked, the most confident first (smaller S_q, ties to the lower position);
+     *   2 random remasking: every masked position of the current block is unmasked with probability 1 / k_b, drawn from
+     *     Philox-4x32-10 with key = seed, counter = (response position, step index N - k, sequence index, 0): unmask iff
+     *     first output word * k_b < 2^32.
+     * block_len cuts the response into blocks decoded left to right (semi-autoregressive remasking): block j is
+     * [j * block_len, min(L, (j + 1) * block_len)), gets N / n_blocks steps (N must be a multiple of n_blocks), and L_b,
+     * N_b, k_b are the block's own length, step count and countdown.  block_len 0 (or >= gen_len) is one block.
+     * The SlowFast hyper-parameters above are ignored by samplers 1 and 2.  Their d_trace record is
+     * (block, block start, block end, k_b, 0, n_sel, n_masked_after, k_remaining_after). */
+    int32_t sampler;          /* 0 */
+    int32_t block_len;        /* 0 */
+    uint32_t seed_lo, seed_hi;/* 0     64-bit seed of random remasking */
 } sfs_params;
 
 /* Per-sequence scheduler state, device-resident, plain data (Algorithm 1's k, s_cycle, e_cycle, H_W, step_count). */

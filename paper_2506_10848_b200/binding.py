@@ -14,6 +14,7 @@ SFS_OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_OOM, ERR_STEP_LIMIT, ERR_TIMEOUT, ERR_MISSING_ROW = -1, -2, -3, -4, -5, -6, -7
 LOGITS_BF16, LOGITS_F32 = 0, 1
 PHASE_SLOW, PHASE_FAST = 0, 1
+SAMPLER_SLOWFAST, SAMPLER_LOW_CONFIDENCE, SAMPLER_RANDOM = 0, 1, 2
 CONF_QBITS = 28
 MAX_W_HIST = 8
 TRACE_INTS = 8
@@ -32,11 +33,15 @@ class Weights(Structure):
 class Params(Structure):
     _fields_ = [("tau_min_conf", c_float), ("tau_high_conf", c_float), ("sigma2_stable", c_float),
                 ("k_max", c_int32), ("w_hist", c_int32), ("k_slow", c_int32), ("k_fast", c_int32),
-                ("max_steps", c_int32), ("min_high_count", c_int32)]
+                ("max_steps", c_int32), ("min_high_count", c_int32),
+                ("sampler", c_int32), ("block_len", c_int32), ("seed_lo", ctypes.c_uint32), ("seed_hi", ctypes.c_uint32)]
 
     @staticmethod
     def default(**kw):
-        p = Params(0.1, 0.85, 1.0, 8, 2, 1, 1, 0, 1)
+        p = Params(0.1, 0.85, 1.0, 8, 2, 1, 1, 0, 1, 0, 0, 0, 0)
+        if "seed" in kw:
+            seed = int(kw.pop("seed"))
+            kw["seed_lo"], kw["seed_hi"] = seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF
         for k, v in kw.items():
             setattr(p, k, v)
         return p

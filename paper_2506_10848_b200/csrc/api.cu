@@ -24,9 +24,18 @@ void set_error(const char *fmt, ...)
     va_end(ap);
 }
 
-static int32_t check_params(const sfs_params *p)
+// gen_len < 0: the response length is not known to the caller of this check
+static int32_t check_params(const sfs_params *p, int32_t gen_len = -1)
 {
     SFS_REQUIRE(p != nullptr, SFS_ERR_INVALID_ARG, "params is NULL");
+    SFS_REQUIRE(p->sampler >= SFS_SAMPLER_SLOWFAST && p->sampler <= SFS_SAMPLER_RANDOM, SFS_ERR_INVALID_ARG, "sampler %d", p->sampler);
+    SFS_REQUIRE(p->block_len >= 0, SFS_ERR_INVALID_ARG, "block_len %d must be >= 0", p->block_len);
+    if (p->sampler != SFS_SAMPLER_SLOWFAST && gen_len > 0) {
+        const int N = p->max_steps > 0 ? p->max_steps : gen_len;
+        const int bl = (p->block_len > 0 && p->block_len < gen_len) ? p->block_len : gen_len;
+        const int nb = (gen_len + bl - 1) / bl;
+        SFS_REQUIRE(N % nb == 0, SFS_ERR_INVALID_ARG, "max_steps %d must be a multiple of the %d blocks of %d positions", N, nb, bl);
+    }
     SFS_REQUIRE(p->w_hist >= 1 && p->w_hist <= SFS_MAX_W_HIST, SFS_ERR_INVALID_ARG, "w_hist %d outside [1, %d]", p->w_hist, SFS_MAX_W_HIST);
     SFS_REQUIRE(p->k_max >= 1, SFS_ERR_INVALID_ARG, "k_max %d must be >= 1", p->k_max);
     SFS_REQUIRE(p->k_slow >= 1 && p->k_fast >= 1, SFS_ERR_INVALID_ARG, "k_slow / k_fast must be >= 1");
@@ -545,7 +554,7 @@ int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab,
 int32_t sfs_state_init(sfs_state *d_state, int32_t B, int32_t gen_len, const sfs_params *params, void *stream)
 {
     SFS_REQUIRE(d_state != nullptr && B >= 1 && gen_len >= 0, SFS_ERR_INVALID_ARG, "state_init: bad arguments");
-    int32_t rc = check_params(params);
+    int32_t rc = check_params(params, gen_len);
     if (rc != SFS_OK) return rc;
     return launch_state_init(d_state, B, gen_len, *params, nullptr, (cudaStream_t)stream);
 }
@@ -566,7 +575,7 @@ int32_t sfs_select(sfs_session *s, const void *d_logits, int32_t logits_dtype, i
     SFS_REQUIRE(logits_dtype == SFS_LOGITS_BF16 || logits_dtype == SFS_LOGITS_F32, SFS_ERR_INVALID_ARG, "logits_dtype %d", logits_dtype);
     const int32_t vocab = s->vocab;
     SFS_REQUIRE(ld >= vocab, SFS_ERR_INVALID_ARG, "ld %lld < vocab %d", (long long)ld, vocab);
-    int32_t rc = check_params(params);
+    int32_t rc = check_params(params, S - P);
     if (rc != SFS_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     rc = launch_row_stats(d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, d_rows, nullptr, nullptr, nullptr,
@@ -661,7 +670,7 @@ int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, i
     SFS_REQUIRE(B >= 1 && B <= s->max_batch && P >= 0 && gen_len >= 1 && P + gen_len <= s->max_seq, SFS_ERR_INVALID_ARG,
                 "generate: B=%d P=%d gen_len=%d outside the session's limits (%d, %d)", B, P, gen_len, s->max_batch, s->max_seq);
     SFS_REQUIRE(P == 0 || d_prompt != nullptr, SFS_ERR_INVALID_ARG, "generate: d_prompt is NULL");
-    int32_t rc = check_params(params);
+    int32_t rc = check_params(params, gen_len);
     if (rc != SFS_OK) return rc;
     const int S = P + gen_len;
     if ((rc = session_plan(s, B, S)) != SFS_OK) return rc;

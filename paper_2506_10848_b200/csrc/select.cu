@@ -1,4 +1,5 @@
-// The SlowFast transition rule S (paper Section 3.3, Algorithm 1), one denoising step, on the device.
+// The transition rule S of one denoising step, on the device: the SlowFast rule (paper Section 3.3, Algorithm 1) or one of
+// the LLaDA strategies of Section 3.1 (low-confidence / random remasking, optionally block by block).
 // One CTA per sequence: it reads the row statistics the epilogue scattered by token position, applies the
 // exploratory (slow) or accelerated (fast) rule, unmasks the chosen positions in place, advances the
 // per-sequence state (k, s_cycle, e_cycle, H_W, phase) and lists the rows the next step needs.  The last CTA
@@ -55,7 +56,37 @@ __device__ int block_sum(int v, int *s_tmp) {
     return r;
 }
 
-enum { MODE_ALL = 0, MODE_TOPK = 1, MODE_HIGH = 2 };
+enum { MODE_ALL = 0, MODE_TOPK = 1, MODE_HIGH = 2, MODE_RANDOM = 3 };
+
+// Philox-4x32-10 (Salmon et al., SC'11): ten rounds of multiply / xor on a 128-bit counter under a 64-bit key; the first
+// output word is returned.  Random remasking draws one word per (position, step, sequence).
+__device__ __forceinline__ uint32_t philox_first_word(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1)
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+        const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+        c0 = h1 ^ c1 ^ k0; c1 = l1; c2 = h0 ^ c3 ^ k1; c3 = l0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return c0;
+}
+
+// block structure of the LLaDA strategies: which positions the step with index t works on, and the block's countdown
+struct BlockStep { int j, lo, hi, k_b, steps_per_block; };
+__device__ __forceinline__ BlockStep block_step(const sfs_params &p, int L, int t)
+{
+    const int N = p.max_steps > 0 ? p.max_steps : L;
+    const int bl = (p.block_len > 0 && p.block_len < L) ? p.block_len : max(L, 1);
+    const int nb = (L + bl - 1) / bl;
+    BlockStep s;
+    s.steps_per_block = max(N / max(nb, 1), 1);
+    s.j = t / s.steps_per_block;
+    s.k_b = s.steps_per_block - (t - s.j * s.steps_per_block);
+    s.lo = min(L, s.j * bl);
+    s.hi = min(L, s.lo + bl);
+    return s;
+}
 
 // dynamic shared memory: keys u64[L] | flags u8[L] (selected) | flags u8[L] (above tau_high)
 __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
@@ -78,14 +109,17 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
     const sfs_params &p = a.params;
 
     const bool active = !st.done && st.status == SFS_OK;
+    const bool vanilla = p.sampler != SFS_SAMPLER_SLOWFAST;
     int n_sel = 0, e_cand = -1, stable = 0;
-    const int rec_phase = st.phase, rec_s = st.s_cycle;
+    int rec_phase = st.phase, rec_s = st.s_cycle;
     int rec_hi = (st.phase == SFS_PHASE_SLOW) ? L : st.hi;
+    const BlockStep blk = block_step(p, L, st.steps_done);
+    if (vanilla) { rec_phase = blk.j; rec_s = blk.lo; rec_hi = blk.hi; e_cand = blk.k_b; }
 
     if (active) {
-        const bool forced = (st.k_remaining == 1);
-        const int lo = forced ? 0 : st.s_cycle;
-        const int hi = forced ? L : ((st.phase == SFS_PHASE_SLOW) ? L : st.hi);
+        const bool forced = !vanilla && (st.k_remaining == 1);
+        const int lo = vanilla ? blk.lo : (forced ? 0 : st.s_cycle);
+        const int hi = vanilla ? blk.hi : (forced ? L : ((st.phase == SFS_PHASE_SLOW) ? L : st.hi));
 
         // ---- candidates of this step and their statistics
         BlockRed r{0, 0, -1, 0x7FFFFFFF, 0, 0};
@@ -108,12 +142,18 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
         }
         r = block_reduce(r, s_tmp);
 
-        if (r.missing > 0 || r.n_cand == 0) {
+        if (r.missing > 0 || (r.n_cand == 0 && !vanilla)) {
             // a needed row was not supplied (or the state is inconsistent): report, change nothing
             if (tid == 0) st.status = SFS_ERR_MISSING_ROW;
         } else {
             int mode, k_top = 0;
-            if (forced) mode = MODE_ALL;
+            if (p.sampler == SFS_SAMPLER_LOW_CONFIDENCE) {
+                // Section 3.1: after this step floor(L_b (1 - (k_b - 1) / N_b)) positions of the block are unmasked
+                const long long Lb = hi - lo, Nb = blk.steps_per_block;
+                const long long target = (Lb * (Nb - blk.k_b + 1)) / Nb;
+                mode = MODE_TOPK; k_top = (int)max(0ll, target - (Lb - r.n_cand));
+            } else if (p.sampler == SFS_SAMPLER_RANDOM) mode = MODE_RANDOM;
+            else if (forced) mode = MODE_ALL;
             else if (st.phase == SFS_PHASE_SLOW) { mode = MODE_TOPK; k_top = p.k_slow; }
             else if (r.n_high >= p.min_high_count) mode = MODE_HIGH;
             else { mode = MODE_TOPK; k_top = p.k_fast; }
@@ -126,6 +166,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
                 bool sel;
                 if (mode == MODE_ALL) sel = true;
                 else if (mode == MODE_HIGH) sel = s_high[i] != 0;
+                else if (mode == MODE_RANDOM)
+                    sel = (unsigned long long)philox_first_word((uint32_t)i, (uint32_t)st.steps_done, (uint32_t)b, 0u, p.seed_lo, p.seed_hi)
+                          * (unsigned long long)blk.k_b < (1ull << 32);
                 else {
                     int rank = 0;                           // candidates that are more confident (ties: smaller position)
                     for (int j = 0; j < L; ++j) rank += (s_keys[j] < key) ? 1 : 0;
@@ -139,7 +182,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
             if (tid == 0) {
                 st.n_masked = r.n_masked - n_sel;
                 st.steps_done++;
-                if (forced) {
+                if (vanilla) {
+                    st.k_remaining--;
+                } else if (forced) {
                     st.k_remaining = 0;
                 } else if (st.phase == SFS_PHASE_SLOW) {
                     e_cand = (r.max_above >= 0) ? r.max_above : r.min_cand;
@@ -164,7 +209,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
             __syncthreads();
 
             // ---- is the span clean?  (decides whether the next cycle starts)
-            if (!forced && st.phase == SFS_PHASE_FAST) {
+            if (!vanilla && !forced && st.phase == SFS_PHASE_FAST) {
                 int cnt = 0;
                 for (int i = st.s_cycle + tid; i < st.hi && i < L; i += kSelThreads) cnt += msk[i] ? 1 : 0;
                 cnt = block_sum(cnt, s_tmp);
@@ -190,9 +235,10 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
     // ---- ordered outputs (warp 0: ballot scan): selected positions, and the rows of the next step
     if (tid < 32) {
         const bool next_active = !st.done && st.status == SFS_OK;
-        const bool nforced = st.k_remaining == 1;
-        const int nlo = nforced ? 0 : st.s_cycle;
-        const int nhi = nforced ? L : ((st.phase == SFS_PHASE_SLOW) ? L : st.hi);
+        const bool nforced = !vanilla && st.k_remaining == 1;
+        const BlockStep nblk = block_step(p, L, st.steps_done);
+        const int nlo = vanilla ? nblk.lo : (nforced ? 0 : st.s_cycle);
+        const int nhi = vanilla ? nblk.hi : (nforced ? L : ((st.phase == SFS_PHASE_SLOW) ? L : st.hi));
         int n_out = 0, n_next = 0;
         for (int base = 0; base < L; base += 32) {
             const int i = base + tid;

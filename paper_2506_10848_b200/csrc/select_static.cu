@@ -80,6 +80,13 @@ extern "C" int32_t sfs_select_static(int32_t vocab, const void *d_logits, int32_
     SFS_REQUIRE(params->w_hist >= 1 && params->w_hist <= SFS_MAX_W_HIST && params->k_max >= 1 && params->k_slow >= 1 &&
                 params->k_fast >= 1 && params->max_steps >= 0 && params->min_high_count >= 1, SFS_ERR_INVALID_ARG,
                 "select_static: hyper-parameters out of range");
+    SFS_REQUIRE(params->sampler >= SFS_SAMPLER_SLOWFAST && params->sampler <= SFS_SAMPLER_RANDOM && params->block_len >= 0,
+                SFS_ERR_INVALID_ARG, "select_static: sampler %d / block_len %d", params->sampler, params->block_len);
+    if (params->sampler != SFS_SAMPLER_SLOWFAST && S > P) {
+        const int L = S - P, N = params->max_steps > 0 ? params->max_steps : L;
+        const int bl = (params->block_len > 0 && params->block_len < L) ? params->block_len : L;
+        SFS_REQUIRE(N % ((L + bl - 1) / bl) == 0, SFS_ERR_INVALID_ARG, "select_static: max_steps %d is not a multiple of the number of blocks", N);
+    }
     StaticScratch *sc = nullptr;
     int32_t rc = scratch_for_current_device(&sc);
     if (rc != SFS_OK) return rc;
