@@ -48,6 +48,12 @@ class SlowFastParams:
     k_fast: int = 1
     max_steps: int = 0             # N; 0 means N = L
     min_high_count: int = 1
+    # Alternative readings of the passages where the paper is at odds with itself, honoured by `slowfast_loop` only (the
+    # step machine, and every other implementation, use the defaults):
+    e_cycle_rule: str = "floor_mean"   # R2: "floor_mean" (equation, Algorithm 1) or "last_candidate" (the prose after it)
+    reset_history: bool = True         # R5: False keeps H_W across cycles, as Algorithm 1 initialises it only once
+    fast_single_step: bool = False     # R6: True takes ONE accelerated step per cycle, as Algorithm 1 prints it; masked
+                                       #     positions left behind s_cycle are then never revisited before the last step
 
 
 def _f32(x: float) -> float:
@@ -102,6 +108,7 @@ class _Sampler:
         self.y: List[Optional[int]] = [None] * L
         self.k = p.max_steps if p.max_steps > 0 else L          # Algorithm 1, initialisation: k = N
         self.trace: List[StepRecord] = []
+        self.H_kept: List[int] = []
 
     def open_positions(self, lo: int, hi: int) -> List[int]:
         return [i for i in range(lo, hi) if self.masked[i]]
@@ -125,10 +132,10 @@ class _Sampler:
         """Section 3.3, exploratory stage from window start s.  Returns the span end hi = e_cycle + 1, or None when
         the sequence (or the budget) ended inside the stage."""
         p, L = self.p, self.L
-        H: List[int] = []                                         # R5: a fresh history per stage
+        H: List[int] = [] if p.reset_history else self.H_kept     # R5: a fresh history per stage
         e_cand = -1
         for _ in range(p.k_max):
-            if self.k == 0 or not any(self.masked):
+            if self.k == 0 or not any(self.masked) or not self.open_positions(s, L):
                 return None
             if self.k == 1:
                 self.last_step(SLOW, s, L)
@@ -138,9 +145,12 @@ class _Sampler:
             reach = [i for i in M if exceeds(sq[i], p.tau_min_conf)]
             e_cand = reach[-1] if reach else M[0]                 # end point of convergence; R3 when nothing reaches tau_min
             H = (H + [e_cand])[-p.w_hist:]
+            self.H_kept = H
             stable = len(H) >= p.w_hist and variance_below(H, p.sigma2_stable)
             self.commit(SLOW, s, L, e_cand, stable, top_k(M, sq, p.k_slow), a)
             if stable:
+                if p.e_cycle_rule == "last_candidate":
+                    return e_cand + 1
                 return sum(H) // len(H) + 1                       # R2: floor of the window's mean
         return e_cand + 1                                         # K_max steps without stability (Algorithm 1's fallback)
 
@@ -156,6 +166,8 @@ class _Sampler:
             high = [i for i in F if exceeds(sq[i], p.tau_high_conf)]
             chosen = high if len(high) >= p.min_high_count else top_k(F, sq, p.k_fast)
             self.commit(FAST, s, hi, -1, False, chosen, a)
+            if p.fast_single_step:
+                return
 
 
 def slowfast_loop(L: int, predict: Predict, p: SlowFastParams) -> Tuple[List[Optional[int]], List[StepRecord]]:
@@ -164,6 +176,10 @@ def slowfast_loop(L: int, predict: Predict, p: SlowFastParams) -> Tuple[List[Opt
     run = _Sampler(L, predict, p)
     s_cycle = 0
     while run.k > 0 and any(run.masked):                          # R7
+        if not run.open_positions(s_cycle, L):
+            # only reachable under fast_single_step: the window has run off the end with masks left behind it;
+            # Algorithm 1 as printed stops here (s_cycle >= L) and returns a sequence that still holds masks
+            break
         hi = run.explore(s_cycle)
         if hi is None or run.k == 0 or not any(run.masked):
             break
@@ -208,6 +224,7 @@ def slowfast_step(st: SlowFastState, a: Dict[int, int], sq: Dict[int, int], p: S
     """Apply one denoising step's decisions to `st` in place.  `a`, `sq` cover rows_needed(st)."""
     if st.done:
         return None
+    assert p.e_cycle_rule == "floor_mean" and p.reset_history and not p.fast_single_step, "the step machine takes the default readings"
     L = st.L
     rec_step = st.steps_done
     if st.k == 1:

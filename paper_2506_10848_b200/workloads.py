@@ -131,3 +131,32 @@ def span(L: int, seed: int):
 def bf16_bits(t: torch.Tensor):
     """bf16 tensor -> numpy uint16 array of its bit patterns (what the oracle's bf16 entry takes)."""
     return t.detach().to("cpu").contiguous().view(torch.int16).numpy().view("uint16")
+
+
+def frontier_confidences(masked, step: int, seed: int, reach: float = 12.0, noise: float = 0.06, seq: int = 0) -> torch.Tensor:
+    """A synthetic confidence process with the shape the paper describes for trained models: positions just behind the
+    decoded frontier are predicted with high confidence, confidence decays with the distance from it, and it jitters
+    from step to step.  masked: sequence of bools; returns float64 [L] in (0.001, 0.999) (1.0 at decoded positions)."""
+    L = len(masked)
+    g = _gen(seed, f"frontier.{seq}.{step}", "cpu")
+    jitter = (torch.rand(L, generator=g, dtype=torch.float64) * 2 - 1) * noise
+    c = torch.ones(L, dtype=torch.float64)
+    open_ = [i for i in range(L) if masked[i]]
+    if open_:
+        front = open_[0]
+        for rank, i in enumerate(open_):
+            d = 0.5 * (i - front) + 0.5 * rank             # distance from the frontier, decoded gaps count half
+            c[i] = min(0.999, max(0.001, 0.97 * float(torch.exp(torch.tensor(-d / reach, dtype=torch.float64))) + float(jitter[i])))
+    return c
+
+
+def logits_for_confidences(conf: torch.Tensor, vocab: int, seed: int, step: int = 0) -> torch.Tensor:
+    """bf16 logits [len(conf), vocab] whose softmax maximum is (up to bf16 rounding of the one non-zero logit) conf[i]:
+    all entries 0 except one winner per row at log(c (V-1) / (1-c)), at a seeded column."""
+    n = conf.numel()
+    g = _gen(seed, f"conf_logits.{step}", "cpu")
+    col = torch.randint(0, vocab, (n,), generator=g)
+    x = torch.zeros((n, vocab), dtype=torch.float32)
+    c = conf.to(torch.float64).clamp(1.0 / vocab + 1e-6, 1 - 1e-9)
+    x[torch.arange(n), col] = torch.log(c * (vocab - 1) / (1 - c)).to(torch.float32)
+    return x.to(torch.bfloat16)
