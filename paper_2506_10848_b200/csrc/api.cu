@@ -362,7 +362,13 @@ __global__ void generate_init_kernel(const int32_t *prompt, int32_t *tokens, uin
     }
 }
 
-__global__ void mirror_active_kernel(const int32_t *ctrl_active, int32_t *host_active) { *host_active = *ctrl_active; }
+// host_active[0]: sequences still decoding; host_active[1]: denoising steps the device has finished in this generation
+__global__ void mirror_active_kernel(const int32_t *ctrl_active, int32_t *host_active, int32_t steps_done)
+{
+    host_active[1] = steps_done;
+    __threadfence_system();
+    host_active[0] = *ctrl_active;
+}
 
 }  // namespace sfs
 
@@ -691,7 +697,7 @@ int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, i
     s->gen_params = *params;
     s->cache_t = 0;                                          // a new generation starts with a full refresh
     s->generating = true;
-    *s->host_active = B;
+    s->host_active[0] = B; s->host_active[1] = 0;
     return SFS_OK;
 }
 
@@ -733,7 +739,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         a.ticket = s->ticket;
         a.trace = (d_trace && s->gen_steps < max_trace_steps) ? d_trace + (size_t)s->gen_steps * B * SFS_TRACE_INTS : nullptr;
         if ((rc = timed_launch(s, SFS_K_SELECT, st, [&] { return launch_select(a, st); })) != SFS_OK) return rc;
-        mirror_active_kernel<<<1, 1, 0, st>>>(s->ctrl + 2, s->host_active_dev);
+        mirror_active_kernel<<<1, 1, 0, st>>>(s->ctrl + 2, s->host_active_dev, s->gen_steps + 1);
         SFS_LAUNCH_CHECK();
         s->launches++;
         s->gen_cur = nxt;
@@ -769,12 +775,21 @@ int32_t sfs_generate(sfs_session *s, const int32_t *d_prompt, int32_t B, int32_t
                      const sfs_params *params, int32_t *d_out_tokens, sfs_state *d_state_out,
                      int32_t *d_trace, int32_t max_trace_steps, void *stream)
 {
+    // the pinned mirror must not receive values of an earlier generation whose kernels are still in flight
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) { set_error("generate: the stream is in an error state"); return SFS_ERR_CUDA; }
     int32_t rc = sfs_generate_begin(s, d_prompt, B, P, gen_len, params, stream);
     if (rc != SFS_OK) return rc;
-    // Steps are enqueued ahead of the device; the pinned mirror of the active-sequence count stops the
-    // enqueueing soon after the last sequence finishes, and kernels of surplus steps exit at once.
+    // Steps are enqueued at most kAhead ahead of the device (enough to keep it busy: a step's launches are enqueued in a
+    // fraction of the time the step runs); the pinned mirror of the active-sequence count stops the enqueueing when the
+    // last sequence finishes, so at most kAhead surplus steps are ever enqueued, and their kernels exit at once.
+    constexpr int kAhead = 2;
+    volatile int32_t *mirror = reinterpret_cast<volatile int32_t *>(s->host_active);
     while (s->gen_steps < s->gen_max_steps) {
-        if (*reinterpret_cast<volatile int32_t *>(s->host_active) == 0) break;
+        long long spins = 0;
+        while (mirror[0] != 0 && s->gen_steps - mirror[1] >= kAhead) {
+            if (++spins > (1ll << 34) || ((spins & 0xFFFFF) == 0 && cudaStreamQuery((cudaStream_t)stream) == cudaSuccess)) break;   // the stream drained or stalled
+        }
+        if (mirror[0] == 0) break;
         if ((rc = sfs_generate_steps(s, 1, d_trace, max_trace_steps, nullptr, nullptr, nullptr, stream)) != SFS_OK) return rc;
     }
     int32_t act = 0;

@@ -183,15 +183,32 @@ def test_batch_of_eight_logits_match_the_oracle_at_the_8b_shape(model8b):
 
 
 def test_cached_steps_match_the_oracle_at_the_8b_shape_under_the_same_schedule(model8b):
-    """Prompt 1024 + 512 masked with the feature cache: one refresh step, one slow partial step and one fast partial step
-    (candidates = the span).  The oracle runs the same schedule in fp32 and is handed the rows the GPU chose; the row
-    choice itself is checked against the oracle's rule applied to the GPU's own similarities (an integer decision)."""
-    from oracle import cache as C
+    """Prompt 1024 + 512 masked with the feature cache at (K_p, K_r) = (100, 8), all 32 layers."""
     shape, w, model = model8b
-    B, P, L = 1, 1024, 512
+    cached_steps_check(shape, w, model, 1024, 512, 100, 8)
+
+
+def test_cached_steps_with_the_long_response_and_the_second_table_4_setting():
+    """The long response (1024 + 1024 tokens: 16 key tiles, 256 recomputed rows) at (K_p, K_r) = (500, 30), on the 8B-width
+    model cut to 4 layers so that the oracle's full-refresh step stays affordable."""
+    shape = W.with_layers(W.LLADA_8B, 4)
+    w = W.model_weights(shape, seed=3, device=DEV)
+    model = sfs.Model(shape, w)
+    try:
+        cached_steps_check(shape, w, model, 1024, 1024, 500, 30)
+    finally:
+        model.close()
+
+
+def cached_steps_check(shape, w, model, P, L, kp, kr):
+    """One refresh step, one slow partial step and one fast partial step (candidates = the span).  The oracle runs the same
+    schedule in fp32 and is handed the rows the GPU chose; the row choice itself is checked against the oracle's rule applied
+    to the GPU's own similarities (an integer decision)."""
+    from oracle import cache as C
+    B = 1
     S = P + L
     nl = shape.n_layers
-    kp, kr, rho = 100, 8, 0.25
+    rho = 0.25
     g = np.random.default_rng(3)
     tok = np.full((B, S), shape.mask_id, dtype=np.int32)
     tok[:, :P] = W.prompt_ids(B, P, shape.vocab - 2, seed=3).numpy()
@@ -201,7 +218,7 @@ def test_cached_steps_match_the_oracle_at_the_8b_shape_under_the_same_schedule(m
     cache = C.FeatureCache(cfg, S, dtype=np.float32)
     rows = [P, P + 1, P + 130, P + 255, S - 1, 17]
     n_adapt = C.adaptive_count(rho, L)
-    span = (120, 200)
+    span = (120, 200) if L == 512 else (300, 700)
     session = sfs.sfs_session_create(model, B, S)
     try:
         sfs.sfs_cache_enable(session, kp, kr, rho)
