@@ -252,7 +252,12 @@ def run_epilogue(torch, sfs, W, shape, dev, peaks):
     arg = torch.empty(R, dtype=torch.int32, device=dev); sq = torch.empty(R, dtype=torch.int64, device=dev)
     rs = lambda i: sfs.sfs_row_stats(bufs[i % 4], sfs.LOGITS_BF16, V, V, None, R, argmax=arg, sq=sq)
     time_back_to_back(torch, rs, 8)
-    us = time_back_to_back(torch, rs, 32) * 1e3
+    us_canonical = time_back_to_back(torch, rs, 32) * 1e3
+    # the pass that streams the logits from HBM inside sfs_select / sfs_generate: exact argmax + enclosure of S_q per row
+    lo_b = torch.empty(R, dtype=torch.int64, device=dev); hi_b = torch.empty(R, dtype=torch.int64, device=dev)
+    rb = lambda i: sfs.sfs_row_stats_bounds(bufs[i % 4], V, V, None, R, lo_b, hi_b, arg)
+    time_back_to_back(torch, rb, 8)
+    us = time_back_to_back(torch, rb, 32) * 1e3
     # one slow and one fast selection step on those logits (row statistics + transition rule)
     ssel = sfs.sfs_select_session_create(V, 1, R)
     rows = torch.arange(R, dtype=torch.int32, device=dev)
@@ -270,13 +275,40 @@ def run_epilogue(torch, sfs, W, shape, dev, peaks):
         torch.cuda.synchronize()
         return time_back_to_back(torch, lambda j: sfs.sfs_select(ssel, bufs[(i + j) % 4], sfs.LOGITS_BF16, V, rows, None, R, tok, msk, 1, R, 0, st,
                                                                   params, sel_count=cnt), 1) * 1e3
+
+    def sel_chain(fast, n=12):
+        """n complete selection steps back to back on cold logits (fresh state each: the same decision every time)."""
+        sts, toks, msks = [], [], []
+        for _ in range(n):
+            tok = torch.full((1, R), shape.mask_id, dtype=torch.int32, device=dev); msk = torch.ones((1, R), dtype=torch.uint8, device=dev)
+            st = torch.zeros((1, sfs.STATE_INTS), dtype=torch.int32, device=dev)
+            sfs.sfs_state_init(st, 1, R, params)
+            if fast:
+                row = st[0].cpu(); row[sfs.STATE_FIELDS.index("phase")] = 1; row[sfs.STATE_FIELDS.index("s_cycle")] = lo
+                row[sfs.STATE_FIELDS.index("hi")] = hi; st[0] = row.to(dev)
+            sts.append(st); toks.append(tok); msks.append(msk)
+        cnt = torch.zeros(1, dtype=torch.int32, device=dev)
+        torch.cuda.synchronize()
+        return time_back_to_back(torch, lambda j: sfs.sfs_select(ssel, bufs[j % 4], sfs.LOGITS_BF16, V, rows, None, R, toks[j], msks[j], 1, R, 0,
+                                                                  sts[j], params, sel_count=cnt), n) * 1e3
     sel_step(0, False)
     slow_us, fast_us = sel_step(1, False), sel_step(2, True)
+    sel_chain(False, 4)
+    slow_chain_us, fast_chain_us = sel_chain(False), sel_chain(True)
     sfs.sfs_session_destroy(ssel)
     gbs = R * V * 2 / us * 1e-3
     out["epilogue"] = {"workload": f"bf16 logits [{R}, {V}], planted winners, seed 1; cold (4 rotating copies > L2)", "row_stats_us": us,
-                       "hbm_gbs": gbs, "frac_of_measured_hbm_peak": gbs / peaks["hbm_gbs"], "select_slow_step_us": slow_us,
-                       "select_fast_step_us": fast_us, "span": [lo, hi]}
+                       "hbm_gbs": gbs, "frac_of_measured_hbm_peak": gbs / peaks["hbm_gbs"],
+                       "kernel": "rowstats_bounds_bf16: the one pass over HBM of the selection step (exact argmax, enclosure of S_q); rows whose "
+                                 "enclosure leaves the step's comparisons open are recomputed canonically from L2 by a second launch",
+                       "canonical_all_rows_us": us_canonical, "canonical_all_rows_hbm_gbs": R * V * 2 / us_canonical * 1e-3,
+                       "select_slow_step_us": slow_us, "select_fast_step_us": fast_us,
+                       "select_slow_step_enqueue_bound_us": slow_chain_us, "select_fast_step_enqueue_bound_us": fast_chain_us,
+                       "select_step_note": "whole sfs_select call (four launches: streaming pass, decision, canonical recompute of the listed rows, "
+                                           "selection): one call timed alone, launch latency included; and 12 calls enqueued back to back, which is "
+                                           "bound by the host's enqueue rate through the Python binding, not by the device (per-kernel device times: "
+                                           "profiles/select_step_256x126464.md)",
+                       "span": [lo, hi]}
     del bufs
     torch.cuda.empty_cache()
     return out

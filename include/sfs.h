@@ -163,6 +163,15 @@ int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab,
                       const int32_t *d_n_rows, int32_t max_rows,
                       int32_t *d_argmax, uint64_t *d_sq, float *d_conf, void *stream);
 
+/* The first of the two passes sfs_select runs over long bf16 rows (65536 to 163840 entries; other shapes return
+ * SFS_ERR_UNSUPPORTED here and take the all-canonical kernels inside sfs_select): exact argmax, and an enclosure
+ * d_lo[r] <= S_q <= d_hi[r] of the canonical denominator from a cheap pass (special-function exponentials, fp32 sums;
+ * relative width 1.2e-4 plus vocab + 2).  sfs_select recomputes the canonical S_q only for rows whose enclosure leaves a
+ * threshold comparison or the top-1 ranking of the step open, so its decisions are those of all-canonical values.
+ * Exposed for tests and measurements. */
+int32_t sfs_row_stats_bounds(const void *d_logits, int32_t vocab, int64_t ld, const int32_t *d_n_rows, int32_t max_rows,
+                             uint64_t *d_lo, uint64_t *d_hi, int32_t *d_argmax, void *stream);
+
 /* Initial scheduler state for B sequences of gen_len masked positions (Algorithm 1, initialisation). */
 int32_t sfs_state_init(sfs_state *d_state, int32_t B, int32_t gen_len, const sfs_params *params, void *stream);
 

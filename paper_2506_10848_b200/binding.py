@@ -117,6 +117,11 @@ def sfs_row_stats(logits, logits_dtype, vocab, ld, n_rows_dev, max_rows, argmax=
                                c_int32(max_rows), _ptr(argmax), _ptr(sq), _ptr(conf), _stream(stream)))
 
 
+def sfs_row_stats_bounds(logits, vocab, ld, n_rows_dev, max_rows, lo, hi, argmax=None, stream=None):
+    _check(lib().sfs_row_stats_bounds(_ptr(logits), c_int32(vocab), c_int64(ld), _ptr(n_rows_dev), c_int32(max_rows), _ptr(lo), _ptr(hi),
+                                      _ptr(argmax), _stream(stream)))
+
+
 def sfs_state_init(state, B, gen_len, params, stream=None):
     _check(lib().sfs_state_init(_ptr(state), c_int32(B), c_int32(gen_len), byref(params), _stream(stream)))
 

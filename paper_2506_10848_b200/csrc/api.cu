@@ -70,12 +70,41 @@ static int32_t dev_alloc(sfs_session *s, T **out, size_t count, bool zero)
     return SFS_OK;
 }
 
+// Row statistics of one selection step into the session's scratch: the two-pass (filter + exact) form for long bf16 rows,
+// the all-canonical kernels otherwise.  Either way the selection kernel finds, for every supplied row the rule reads, a
+// value in pos_sq that gives the decisions of the canonical S_q.
+static int32_t step_row_stats(sfs_session *s, const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
+                              const int32_t *d_n_rows, int32_t max_rows, const int32_t *d_rows, const uint8_t *d_mask,
+                              int32_t B, int32_t S, int32_t P, const sfs_state *d_state, const sfs_params &params, bool *two_pass,
+                              cudaStream_t st)
+{
+    int32_t *err = device_status_word();
+    *two_pass = row_stats_two_pass_applies(d_logits, logits_dtype, vocab, ld);
+    if (!*two_pass)
+        return launch_row_stats(d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, d_rows, nullptr, nullptr, nullptr,
+                                s->pos_sq, s->pos_arg, B * S, err, st);
+    RefineArgs rf{};
+    rf.mask = d_mask; rf.B = B; rf.S = S; rf.P = P; rf.L = S - P; rf.state = d_state; rf.params = params;
+    rf.pos_lo = s->pos_lo; rf.pos_hi = s->pos_hi; rf.pos_sq = s->pos_sq; rf.pos_arg = s->pos_arg;
+    rf.slice_partials = s->slice_partials; rf.row_tickets = s->row_tickets;
+    rf.pos_row = s->pos_row; rf.pos_max = s->pos_max; rf.refine_list = s->refine_list; rf.refine_count = s->refine_count;
+    return launch_row_stats_two_pass(d_logits, vocab, ld, d_n_rows, max_rows, d_rows, rf, err, st);
+}
+
 static int32_t session_alloc_select(sfs_session *s)
 {
     const size_t n = (size_t)s->max_batch * s->max_seq;
     int32_t rc;
     if ((rc = dev_alloc(s, &s->pos_sq, n, true)) != SFS_OK) return rc;
     if ((rc = dev_alloc(s, &s->pos_arg, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->pos_lo, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->pos_hi, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->slice_partials, n * kRowStatsSlices * 4, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->row_tickets, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->pos_row, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->pos_max, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->refine_list, n, true)) != SFS_OK) return rc;
+    if ((rc = dev_alloc(s, &s->refine_count, 4, true)) != SFS_OK) return rc;
     if ((rc = dev_alloc(s, &s->seq_rows, n, true)) != SFS_OK) return rc;
     if ((rc = dev_alloc(s, &s->seq_row_count, (size_t)s->max_batch, true)) != SFS_OK) return rc;
     if ((rc = dev_alloc(s, &s->ticket, 4, true)) != SFS_OK) return rc;
@@ -557,6 +586,15 @@ int32_t sfs_row_stats(const void *d_logits, int32_t logits_dtype, int32_t vocab,
                             (cudaStream_t)stream);
 }
 
+int32_t sfs_row_stats_bounds(const void *d_logits, int32_t vocab, int64_t ld, const int32_t *d_n_rows, int32_t max_rows,
+                             uint64_t *d_lo, uint64_t *d_hi, int32_t *d_argmax, void *stream)
+{
+    SFS_REQUIRE(d_logits != nullptr && d_lo != nullptr && d_hi != nullptr, SFS_ERR_INVALID_ARG, "row_stats_bounds: NULL pointer");
+    SFS_REQUIRE(vocab >= 1 && vocab < (1 << 19) && ld >= vocab && max_rows >= 0, SFS_ERR_INVALID_ARG, "row_stats_bounds: bad sizes");
+    return launch_row_stats_bounds(d_logits, vocab, ld, d_n_rows, max_rows, reinterpret_cast<unsigned long long *>(d_lo),
+                                   reinterpret_cast<unsigned long long *>(d_hi), d_argmax, device_status_word_if_any(), (cudaStream_t)stream);
+}
+
 int32_t sfs_state_init(sfs_state *d_state, int32_t B, int32_t gen_len, const sfs_params *params, void *stream)
 {
     SFS_REQUIRE(d_state != nullptr && B >= 1 && gen_len >= 0, SFS_ERR_INVALID_ARG, "state_init: bad arguments");
@@ -584,10 +622,11 @@ int32_t sfs_select(sfs_session *s, const void *d_logits, int32_t logits_dtype, i
     int32_t rc = check_params(params, S - P);
     if (rc != SFS_OK) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    rc = launch_row_stats(d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, d_rows, nullptr, nullptr, nullptr,
-                          s->pos_sq, s->pos_arg, B * S, device_status_word(), st);
+    bool two_pass = false;
+    rc = step_row_stats(s, d_logits, logits_dtype, vocab, ld, d_n_rows, max_rows, d_rows, d_mask, B, S, P, d_state, *params, &two_pass, st);
     if (rc != SFS_OK) return rc;
     SelectArgs a{};
+    a.pos_lo = two_pass ? s->pos_lo : nullptr;
     a.tokens = d_tokens; a.mask = d_mask; a.B = B; a.S = S; a.P = P; a.L = S - P;
     a.state = d_state; a.params = *params;
     a.pos_sq = s->pos_sq; a.pos_arg = s->pos_arg;
@@ -727,10 +766,12 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
             if (d_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_rows_dump, rows, (size_t)B * L * 4, cudaMemcpyDeviceToDevice, st));
             if (d_n_rows_dump) SFS_CUDA(cudaMemcpyAsync(d_n_rows_dump, n_rows, 4, cudaMemcpyDeviceToDevice, st));
         }
+        bool two_pass = false;
         if ((rc = timed_launch(s, SFS_K_ROW_STATS, st, [&] {
-                 return launch_row_stats(s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, nullptr, nullptr, nullptr,
-                                         s->pos_sq, s->pos_arg, B * S, err, st); })) != SFS_OK) return rc;
+                 return step_row_stats(s, s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, s->mask, B, S, P, s->state,
+                                       s->gen_params, &two_pass, st); })) != SFS_OK) return rc;
         SelectArgs a{};
+        a.pos_lo = two_pass ? s->pos_lo : nullptr;
         a.tokens = s->tokens; a.mask = s->mask; a.B = B; a.S = S; a.P = P; a.L = L;
         a.state = s->state; a.params = s->gen_params;
         a.pos_sq = s->pos_sq; a.pos_arg = s->pos_arg;

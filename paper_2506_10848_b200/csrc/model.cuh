@@ -25,6 +25,10 @@ struct sfs_session {
     // selection scratch
     unsigned long long *pos_sq = nullptr;    // [max_batch*max_seq]
     int32_t *pos_arg = nullptr;              // [max_batch*max_seq]
+    unsigned long long *pos_lo = nullptr, *pos_hi = nullptr;   // [max_batch*max_seq] enclosures of the two-pass row statistics
+    float *slice_partials = nullptr; int32_t *row_tickets = nullptr;   // scratch of its first pass
+    int32_t *pos_row = nullptr, *refine_list = nullptr, *refine_count = nullptr;   // rows its second pass recomputes
+    float *pos_max = nullptr;                                                       // exact row maximum per position
     int32_t *seq_rows = nullptr;             // [max_batch*max_seq]
     int32_t *seq_row_count = nullptr;        // [max_batch]
     int32_t *ticket = nullptr;               // [1]

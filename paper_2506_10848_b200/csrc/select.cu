@@ -72,22 +72,6 @@ __device__ __forceinline__ uint32_t philox_first_word(uint32_t c0, uint32_t c1, 
     return c0;
 }
 
-// block structure of the LLaDA strategies: which positions the step with index t works on, and the block's countdown
-struct BlockStep { int j, lo, hi, k_b, steps_per_block; };
-__device__ __forceinline__ BlockStep block_step(const sfs_params &p, int L, int t)
-{
-    const int N = p.max_steps > 0 ? p.max_steps : L;
-    const int bl = (p.block_len > 0 && p.block_len < L) ? p.block_len : max(L, 1);
-    const int nb = (L + bl - 1) / bl;
-    BlockStep s;
-    s.steps_per_block = max(N / max(nb, 1), 1);
-    s.j = t / s.steps_per_block;
-    s.k_b = s.steps_per_block - (t - s.j * s.steps_per_block);
-    s.lo = min(L, s.j * bl);
-    s.hi = min(L, s.lo + bl);
-    return s;
-}
-
 // dynamic shared memory: keys u64[L] | flags u8[L] (selected) | flags u8[L] (above tau_high)
 __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
 {
@@ -225,10 +209,11 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
         __syncthreads();
         // the statistics of this step are consumed: a later step must bring its own
         for (int i = tid; i < L; i += kSelThreads) psq[i] = 0;
+        if (a.pos_lo) for (int i = tid; i < L; i += kSelThreads) a.pos_lo[(long long)b * S + P + i] = 0;
     } else {
         // a finished (or stopped) sequence consumes the statistics supplied for it as well: nothing stale is left for a
         // later generation that reuses the scratch
-        for (int i = tid; i < L; i += kSelThreads) { s_sel[i] = 0; psq[i] = 0; }
+        for (int i = tid; i < L; i += kSelThreads) { s_sel[i] = 0; psq[i] = 0; if (a.pos_lo) a.pos_lo[(long long)b * S + P + i] = 0; }
     }
     __syncthreads();
 

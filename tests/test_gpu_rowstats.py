@@ -108,3 +108,49 @@ def test_long_rows_special_values_padding_and_device_row_count():
     assert np.array_equal(arg[:4], ref["argmax"][:4]) and np.array_equal(sq[:4], ref["sq"][:4])
     assert np.all(arg[4:] == -7)
     sfs.sfs_check_device_status()
+
+
+def gpu_bounds(logits, vocab, ld):
+    R = logits.shape[0]
+    lo = torch.zeros(R, dtype=torch.int64, device=DEV); hi = torch.zeros(R, dtype=torch.int64, device=DEV)
+    arg = torch.full((R,), -7, dtype=torch.int32, device=DEV)
+    sfs.sfs_row_stats_bounds(logits, vocab, ld, None, R, lo, hi, arg)
+    torch.cuda.synchronize()
+    return lo.cpu().numpy().view(np.uint64), hi.cpu().numpy().view(np.uint64), arg.cpu().numpy()
+
+
+@pytest.mark.parametrize("V,ld", [(126464, 126464), (65536, 65536 + 64), (131072, 131072)])
+def test_enclosures_of_the_cheap_pass_contain_the_canonical_denominator(V, ld):
+    """The enclosure [lo, hi] that the first pass of the selection's row statistics emits must contain the oracle's canonical
+    S_q for every row — workload-like rows, flat rows (S_q = V 2^28), rows dominated by one logit, rows with -inf entries —
+    and must be narrow (relative width 1.2e-4 plus the truncation allowance V), else the second pass would recompute
+    everything.  Rows the cheap pass cannot bound (infinite or NaN sums) get an enclosure that contains everything."""
+    R = 64
+    x = W.planted_logits(R, V, seed=9, device="cpu").float()
+    g = torch.Generator().manual_seed(V)
+    x[1, :] = 0.5                                           # flat row
+    x[2, :] = -3.0; x[2, 77] = 40.0                         # one logit dominates: S_q = 2^28 exactly
+    x[3, ::2] = -float("inf")                               # half of the row contributes nothing
+    x[4] = torch.randn(V, generator=g) * 0.3                # near-flat: S ~ V, the widest enclosures
+    x[5] = torch.randn(V, generator=g) * 30.0               # very spread
+    x[6, :] = -float("inf"); x[6, 5] = 1.0                  # a single finite entry
+    x[7, :] = -float("inf")                                 # nothing finite: left to the canonical pass
+    x[8, 11] = float("inf")                                 # an infinite maximum: left to the canonical pass
+    full = torch.zeros((R, ld), dtype=torch.bfloat16)
+    full[:, :V] = x.to(torch.bfloat16)
+    ref = RS.row_stats(np.ascontiguousarray(W.bf16_bits(full)[:, :V]))
+    lo, hi, arg = gpu_bounds(full.to(DEV), V, ld)
+    sq = ref["sq"].astype(np.uint64)
+    open_rows = {7, 8}
+    for r in range(R):
+        if r in open_rows:
+            assert lo[r] <= 1 and hi[r] >= (1 << 62), r
+            continue
+        assert arg[r] == ref["argmax"][r], r
+        assert lo[r] <= sq[r] <= hi[r], (r, int(lo[r]), int(sq[r]), int(hi[r]))
+        assert float(hi[r] - lo[r]) <= 1.3e-4 * float(sq[r]) + 2.0 * V + 8, (r, int(hi[r] - lo[r]), int(sq[r]))
+        assert lo[r] >= (1 << 28)
+    # the approximate sum itself is far inside the enclosure: the slack is a safety factor, not a fit
+    mid = (lo.astype(np.float64) + hi.astype(np.float64)) / 2
+    rows = [r for r in range(R) if r not in open_rows]
+    assert np.max(np.abs(mid[rows] - sq[rows].astype(np.float64)) / sq[rows].astype(np.float64)) <= 2e-5 + V / float(1 << 28)

@@ -241,3 +241,47 @@ def test_statistics_of_a_finished_sequence_do_not_survive_into_the_next_generati
         assert state_to_dict(state[0])["status"] == sfs.ERR_MISSING_ROW and int(mask.sum()) == L
     finally:
         sfs.sfs_session_destroy(session)
+
+
+@pytest.mark.parametrize("case", ["near_ties", "threshold_edges", "all_confident"])
+def test_full_vocabulary_steps_where_the_cheap_pass_cannot_decide(case):
+    """Long bf16 rows take the two-pass row statistics.  These inputs are built so that the enclosures of the cheap pass
+    leave the step's questions open — top-1 candidates closer than the enclosure width, confidences within 1e-5 of a
+    threshold, many rows with S_q = 2^28 exactly — and the decisions must still be the oracle's, slow and fast step."""
+    V, L, P, B = 126464, 48, 0, 1
+    po, pg = params_pair()
+    if case == "near_ties":
+        conf = torch.full((L,), 0.05, dtype=torch.float64)
+        conf[10] = 0.30000; conf[20] = 0.30001; conf[30] = 0.29999; conf[31] = 0.30000        # best four within 3e-5 relative
+    elif case == "threshold_edges":
+        conf = torch.linspace(0.02, 0.95, L, dtype=torch.float64)
+        conf[5] = 0.1 + 1e-6; conf[6] = 0.1 - 1e-6; conf[7] = 0.85 + 1e-6; conf[8] = 0.85 - 1e-6; conf[40] = 0.1000001
+    else:
+        conf = torch.full((L,), 1.0 - 1e-12, dtype=torch.float64)
+    logits = W.logits_for_confidences(conf, V, seed=3)
+    stats = RS.row_stats(W.bf16_bits(logits))
+    session = sfs.sfs_select_session_create(V, B, L)
+    try:
+        for phase, span in ((SLOW, None), (FAST, (4, 44))):
+            tokens = torch.full((B, L), V - 1, dtype=torch.int32, device=DEV)
+            mask = torch.ones((B, L), dtype=torch.uint8, device=DEV)
+            state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+            sfs.sfs_state_init(state, B, L, pg)
+            ost = SlowFastState.fresh(L, po)
+            if phase == FAST:
+                write_state(state, 0, phase=1, s_cycle=span[0], hi=span[1])
+                ost.phase, ost.s_cycle, ost.hi = FAST, span[0], span[1]
+            rows = torch.arange(L, dtype=torch.int32, device=DEV)
+            sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+            sel_pos = torch.zeros((B, L), dtype=torch.int32, device=DEV); sel_tok = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+            trace = torch.zeros((B, sfs.TRACE_INTS), dtype=torch.int32, device=DEV)
+            sfs.sfs_select(session, logits.to(DEV), sfs.LOGITS_BF16, V, rows, None, L, tokens, mask, B, L, P, state, pg,
+                           sel_count, sel_pos, sel_tok, trace=trace)
+            torch.cuda.synchronize()
+            rec = slowfast_step(ost, {i: int(stats["argmax"][i]) for i in range(L)}, {i: int(stats["sq"][i]) for i in range(L)}, po)
+            n = int(sel_count[0])
+            assert sel_pos[0, :n].tolist() == rec.positions and sel_tok[0, :n].tolist() == rec.tokens, (case, phase)
+            assert trace[0].tolist()[:6] == [rec.phase, rec.s, rec.hi, rec.e_cand, rec.stable, len(rec.positions)], (case, phase)
+        sfs.sfs_check_device_status()
+    finally:
+        sfs.sfs_session_destroy(session)
