@@ -307,7 +307,7 @@ def run_epilogue(torch, sfs, W, shape, dev, peaks):
                        "select_step_note": "whole sfs_select call (four launches: streaming pass, decision, canonical recompute of the listed rows, "
                                            "selection): one call timed alone, launch latency included; and 12 calls enqueued back to back, which is "
                                            "bound by the host's enqueue rate through the Python binding, not by the device (per-kernel device times: "
-                                           "profiles/select_step_256x126464.md)",
+                                           "profiles/rowstats_bounds_256x126464.md)",
                        "span": [lo, hi]}
     del bufs
     torch.cuda.empty_cache()
