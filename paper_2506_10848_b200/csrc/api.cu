@@ -346,17 +346,17 @@ static int32_t run_body_cached(sfs_session *s, const int32_t *d_tokens, int32_t 
                 if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_cache_select(a, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_gather_rows_bf16(s->h, s->sel_rows, NR, d, s->hg, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_QKV, st, [&] { return gemm_launch(gp.qkv, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-                if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope(s->qk, 2 * d, NR, S, c.n_heads, c.head_dim, s->rope_table, s->sel_rows, st); })) != SFS_OK) return rc;
-                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_kv(s->qk, 2 * d, d, s->vt, T, s->sel_rows, NR, d, s->Kc[l], s->Vtc[l], T, st); })) != SFS_OK) return rc;
+                if ((rc = timed_launch(s, SFS_K_ROPE, st, [&] { return launch_rope_scatter_kv(s->qk, 2 * d, NR, S, c.n_heads, c.head_dim, s->rope_table, s->sel_rows, s->Kc[l], s->vt, T, s->Vtc[l], T, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_ATTENTION, st, [&] { return attn_launch_queries(cl.attn, n_sel, d_active, err, st); })) != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_O, st, [&] { return gemm_launch(gp.o, nullptr, d_active, err, st); })) != SFS_OK) return rc;
-                if ((rc = timed_launch(s, SFS_K_CACHE, st, [&] { return launch_scatter_rows_f32(s->partial, gp.o.args.splits, gp.o.args.split_stride, s->sel_rows, NR, d, s->Ac[l], st); })) != SFS_OK) return rc;
             }
             pend = s->Ac[l]; n_pend = 2;
             if (NR > 0) {
                 const GatherLayerPlans &gp = (*gps)[l];
+                // the O projection's slabs become the attention increments of the recomputed tokens, and the MLP's input rows
                 rc = timed_launch(s, SFS_K_RMSNORM, st, [&] {
-                    return launch_rmsnorm(s->x, s->Ac[l], 1, 0, m->mlp_norm[l], s->hg, s->sel_rows, nullptr, NR, d, c.rms_eps, st);
+                    return launch_fold_norm_rows(s->partial, gp.o.args.splits, gp.o.args.split_stride, s->sel_rows, NR, s->x, s->Ac[l],
+                                                 m->mlp_norm[l], s->hg, d, c.rms_eps, st);
                 });
                 if (rc != SFS_OK) return rc;
                 if ((rc = timed_launch(s, SFS_K_GEMM_GATE_UP, st, [&] { return gemm_launch(gp.gate_up, nullptr, d_active, err, st); })) != SFS_OK) return rc;

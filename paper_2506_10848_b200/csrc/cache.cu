@@ -169,7 +169,135 @@ __global__ void scatter_vt_kernel(const __nv_bfloat16 *__restrict__ vt_src, long
     }
 }
 
+// One launch for what follows the QKV projection of the recomputed rows: the rotary embedding of q and k (in place, on the
+// compact rows; the arithmetic of rope_kernel), the rotated k also written to the token's row of the K cache, and the new
+// value columns scattered into V^T.  Blocks [0, rope_blocks) rotate, the rest scatter values (8 features per block).
+__global__ void __launch_bounds__(256)
+rope_scatter_kv_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int n_rows, int S, int n_heads, int dh, const float2 *__restrict__ table,
+                       const int32_t *__restrict__ rows, __nv_bfloat16 *__restrict__ k_dst, const __nv_bfloat16 *__restrict__ vt_src,
+                       long long ld_vt_src, __nv_bfloat16 *__restrict__ vt_dst, long long ld_vt_dst, int rope_blocks)
+{
+    const int d = n_heads * dh;
+    if ((int)blockIdx.x >= rope_blocks) {
+        const int f0 = ((int)blockIdx.x - rope_blocks) * 8;
+        for (int idx = threadIdx.x; idx < 8 * n_rows; idx += blockDim.x) {
+            const int f = f0 + idx / n_rows, j = idx - (idx / n_rows) * n_rows;
+            if (f < d) vt_dst[(long long)f * ld_vt_dst + rows[j]] = vt_src[(long long)f * ld_vt_src + j];
+        }
+        return;
+    }
+    const int half = dh / 2, groups = half / 8;
+    const unsigned idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned total = (unsigned)n_rows * 2u * (unsigned)n_heads * (unsigned)groups;
+    if (idx >= total) return;
+    const unsigned per_token = (unsigned)groups * 2u * (unsigned)n_heads;
+    const int t = (int)(idx / per_token);
+    const unsigned rem = idx - (unsigned)t * per_token;
+    const int hh = (int)(rem / (unsigned)groups);              // q heads then k heads: contiguous columns
+    const int g = (int)(rem - (unsigned)hh * (unsigned)groups);
+    const int tok = rows[t], pos = tok % S;
+    __nv_bfloat16 *base = qk + (long long)t * ld + (long long)hh * dh + g * 8;
+    uint4 lo = *reinterpret_cast<uint4 *>(base), hi = *reinterpret_cast<uint4 *>(base + half);
+    const float2 *tb = table + (long long)pos * half + g * 8;
+    uint32_t *lw = reinterpret_cast<uint32_t *>(&lo), *hw = reinterpret_cast<uint32_t *>(&hi);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        float x1[2] = {bf16_bits_to_f32(lw[w] & 0xFFFFu), bf16_bits_to_f32(lw[w] >> 16)};
+        float x2[2] = {bf16_bits_to_f32(hw[w] & 0xFFFFu), bf16_bits_to_f32(hw[w] >> 16)};
+        float o1[2], o2[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const float2 cs = tb[2 * w + e];
+            o1[e] = x1[e] * cs.x - x2[e] * cs.y;
+            o2[e] = x2[e] * cs.x + x1[e] * cs.y;
+        }
+        __nv_bfloat162 a = __floats2bfloat162_rn(o1[0], o1[1]), b2 = __floats2bfloat162_rn(o2[0], o2[1]);
+        lw[w] = *reinterpret_cast<uint32_t *>(&a);
+        hw[w] = *reinterpret_cast<uint32_t *>(&b2);
+    }
+    *reinterpret_cast<uint4 *>(base) = lo;
+    *reinterpret_cast<uint4 *>(base + half) = hi;
+    if (hh >= n_heads) {                                       // a key head: also the token's row of the K cache
+        __nv_bfloat16 *kd = k_dst + (long long)tok * d + (long long)(hh - n_heads) * dh + g * 8;
+        *reinterpret_cast<uint4 *>(kd) = lo;
+        *reinterpret_cast<uint4 *>(kd + half) = hi;
+    }
+}
+
+// One launch for what follows the output projection of the recomputed rows: the split-K slabs of compact row j are added in
+// slab order into the attention increment of its token (inc[rows[j]] = sum of slabs), and the MLP branch's input
+// h[j] = bf16(RMSNorm(x[rows[j]] + inc[rows[j]]) * gain) is written to the compact buffer.
+__global__ void __launch_bounds__(256)
+fold_norm_rows_kernel(const float *__restrict__ slabs, int n_slabs, long long slab_stride, const int32_t *__restrict__ rows,
+                      const float *__restrict__ x, float *__restrict__ inc, const __nv_bfloat16 *__restrict__ gain,
+                      __nv_bfloat16 *__restrict__ h, int d, float eps)
+{
+    const int j = blockIdx.x, chunks = d / 4;
+    const long long src = rows[j];
+    const float4 *sp = reinterpret_cast<const float4 *>(slabs + (long long)j * d);
+    const float4 *xr = reinterpret_cast<const float4 *>(x + src * d);
+    float4 *ir = reinterpret_cast<float4 *>(inc + src * d);
+    __shared__ float s_part[8];
+    extern __shared__ float4 s_y[];                            // the row, kept between the two passes
+    float ss = 0.f;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        float4 v = sp[c];
+        for (int k = 1; k < n_slabs; ++k) {
+            const float4 p = sp[(long long)k * (slab_stride / 4) + c];
+            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
+        }
+        ir[c] = v;
+        const float4 xv = xr[c];
+        const float4 y = make_float4(xv.x + v.x, xv.y + v.y, xv.z + v.z, xv.w + v.w);
+        s_y[c] = y;
+        ss += y.x * y.x + y.y * y.y + y.z * y.z + y.w * y.w;
+    }
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) tot += s_part[w];
+    const float inv = rsqrtf(tot / (float)d + eps);
+    const uint2 *gp = reinterpret_cast<const uint2 *>(gain);
+    uint2 *hp = reinterpret_cast<uint2 *>(h + (long long)j * d);
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        const float4 v = s_y[c];
+        const uint2 g = gp[c];
+        __nv_bfloat162 o0 = __floats2bfloat162_rn(v.x * inv * bf16_bits_to_f32(g.x & 0xFFFFu), v.y * inv * bf16_bits_to_f32(g.x >> 16));
+        __nv_bfloat162 o1 = __floats2bfloat162_rn(v.z * inv * bf16_bits_to_f32(g.y & 0xFFFFu), v.w * inv * bf16_bits_to_f32(g.y >> 16));
+        hp[c] = make_uint2(*reinterpret_cast<uint32_t *>(&o0), *reinterpret_cast<uint32_t *>(&o1));
+    }
+}
+
 }  // namespace
+
+int32_t launch_rope_scatter_kv(void *qk, long long ld, int n_rows, int S, int n_heads, int head_dim, const float2 *table, const int32_t *rows,
+                               void *k_dst, const void *vt_src, long long ld_vt_src, void *vt_dst, long long ld_vt_dst, cudaStream_t s)
+{
+    if (n_rows <= 0) return SFS_OK;
+    const long long total = (long long)n_rows * 2 * n_heads * (head_dim / 16);
+    SFS_REQUIRE(total < (1LL << 31), SFS_ERR_INVALID_ARG, "rope: %lld items do not fit a 32-bit index", total);
+    const int rope_blocks = (int)((total + 255) / 256), d = n_heads * head_dim;
+    rope_scatter_kv_kernel<<<rope_blocks + (d + 7) / 8, 256, 0, s>>>(reinterpret_cast<__nv_bfloat16 *>(qk), ld, n_rows, S, n_heads, head_dim, table, rows,
+                                                                      reinterpret_cast<__nv_bfloat16 *>(k_dst), reinterpret_cast<const __nv_bfloat16 *>(vt_src),
+                                                                      ld_vt_src, reinterpret_cast<__nv_bfloat16 *>(vt_dst), ld_vt_dst, rope_blocks);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+int32_t launch_fold_norm_rows(const float *slabs, int n_slabs, long long slab_stride, const int32_t *rows, int n_rows, const float *x, float *inc,
+                              const void *gain, void *h, int d, float eps, cudaStream_t s)
+{
+    if (n_rows <= 0) return SFS_OK;
+    SFS_REQUIRE((size_t)d * 4 <= 96 * 1024, SFS_ERR_UNSUPPORTED, "d_model %d too wide for the fused fold + norm", d);
+    const size_t smem = (size_t)d * 4;
+    if (smem > 48 * 1024) SFS_CUDA(cudaFuncSetAttribute(fold_norm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    fold_norm_rows_kernel<<<n_rows, 256, smem, s>>>(slabs, n_slabs < 1 ? 1 : n_slabs, slab_stride, rows, x, inc, reinterpret_cast<const __nv_bfloat16 *>(gain),
+                                                    reinterpret_cast<__nv_bfloat16 *>(h), d, eps);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
 
 int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld, int d, int t_first, int t_count, int T, float *partial,
                            cudaStream_t s)

@@ -37,4 +37,11 @@ int32_t launch_scatter_rows_f32(const float *src, int n_slabs, long long slab_st
 int32_t launch_scatter_kv(const void *qk_src, long long ld_src, int col0, const void *vt_src, long long ld_vt_src,
                           const int32_t *rows, int n_rows, int d, void *k_dst, void *vt_dst, long long ld_vt_dst, cudaStream_t s);
 
+// rope (as launch_rope, on the compact rows) + rotated k rows into the K cache + new value columns into V^T, one launch
+int32_t launch_rope_scatter_kv(void *qk, long long ld, int n_rows, int S, int n_heads, int head_dim, const float2 *table, const int32_t *rows,
+                               void *k_dst, const void *vt_src, long long ld_vt_src, void *vt_dst, long long ld_vt_dst, cudaStream_t s);
+// inc[rows[j], :] = sum of the slabs of compact row j (slab order); h[j, :] = bf16(RMSNorm(x[rows[j], :] + inc[rows[j], :]) * gain)
+int32_t launch_fold_norm_rows(const float *slabs, int n_slabs, long long slab_stride, const int32_t *rows, int n_rows, const float *x, float *inc,
+                              const void *gain, void *h, int d, float eps, cudaStream_t s);
+
 }  // namespace sfs

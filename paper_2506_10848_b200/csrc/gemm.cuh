@@ -23,6 +23,8 @@ struct GemmArgs {
     int n_per_map;           // rows of each B matrix
     int bn, stages;          // tile width (multiple of 16, <= 256) and depth of the shared-memory ring
     int mb;                  // 256-row blocks per tile (1 or 2)
+    int one_cta;             // 1: tiles of 128 rows computed by single CTAs (few rows: the weights stream through every SM)
+    int tile_rows;           // output rows per tile: mb * 256, or 128
     int n_col_tiles;         // column tiles over all B matrices
     int splits, kb_per_split;        // split-K: the k-blocks are cut into `splits` ranges, range s writes slab s of C
     long long split_stride;          // elements between slabs

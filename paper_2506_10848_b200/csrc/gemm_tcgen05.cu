@@ -89,7 +89,7 @@ __device__ __forceinline__ TileCoord tile_coord(const GemmArgs &g, int tile, int
 {
     TileCoord t;
     const int rest = tile / m_groups;
-    t.m0 = (tile - rest * m_groups) * (g.mb * 2 * BM);     // row groups fastest: pairs that share a weight tile run together
+    t.m0 = (tile - rest * m_groups) * g.tile_rows;         // row groups fastest: pairs that share a weight tile run together
     const int n_tile = rest / g.splits;
     t.split = rest - n_tile * g.splits;
     if (g.mode == GEMM_SWIGLU) {
@@ -414,6 +414,143 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (threadIdx.x == 0 && s_abort && g.err) atomicExch(g.err, SFS_ERR_TIMEOUT);
 }
 
+// ---- few rows (M <= 128): one CTA per tile ------------------------------------------------------------------
+// With at most 128 rows half of a pair's 256-row MMA would multiply padding, and what bounds the projection is streaming the
+// weights: every SM should pull its own slab of weight rows at full rate.  A CTA computes a 128 x BN tile with
+// tcgen05.mma.cta_group::1 (M = 128, N = BN), loading the 128 activation rows and BN weight rows of every k-block itself (the
+// weight rows as two boxes of BN / 2, SwiGLU: gate rows then up rows, so the accumulator layout and the epilogue are those
+// of the pair kernel); BN is chosen so that the tiles fill the SMs in whole waves.  Same warp roles, ring and bounded waits.
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_kernel_1cta(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                 const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
+{
+    if (g.d_active && *g.d_active == 0) return;             // nothing left to decode
+    const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
+    const int m_groups = (M + BM - 1) / BM;
+    const int num_tiles = m_groups * g.n_col_tiles * g.splits;
+    if ((int)blockIdx.x >= num_tiles) return;
+
+    const int BN = g.bn, STAGES = g.stages, HALF = BN >> 1;
+    const int STAGE_BYTES = A_BYTES + BN * BK * 2;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + STAGES * STAGE_BYTES);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * kMaxStages + 4);
+    __shared__ int s_abort;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int num_kb = (g.K + BK - 1) / BK;
+    const uint32_t smem_base = tc::smem_u32(smem);
+    const uint32_t bar_full = tc::smem_u32(bars), bar_empty = bar_full + 8 * kMaxStages;
+    const uint32_t bar_acc_full = bar_full + 16 * kMaxStages, bar_acc_empty = bar_acc_full + 16;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { tc::mbar_init(bar_full + 8 * s, 1); tc::mbar_init(bar_empty + 8 * s, 1); }
+        for (int b = 0; b < 2; ++b) { tc::mbar_init(bar_acc_full + 8 * b, 1); tc::mbar_init(bar_acc_empty + 8 * b, kEpiWarps); }
+        s_abort = 0;
+        tc::mbar_init_fence();
+    }
+    __syncwarp();
+    if (warp == 1) { tc::tmem_alloc(tc::smem_u32(tmem_slot), kTmemCols); tc::tmem_relinquish(); }
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
+    const uint32_t bn_pad = (uint32_t)((BN + 31) & ~31);
+    const uint32_t n_bufs = (uint32_t)g.acc_bufs, buf_stride = 256;
+    const bool swiglu = (g.mode == GEMM_SWIGLU);
+    const int num_ctas = (int)gridDim.x;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) { tc::tma_prefetch_desc(&tmA); tc::tma_prefetch_desc(&tmB0); }
+        uint32_t it = 0;
+        bool ok = true;
+        bool ready = tc::mbar_test(bar_empty, 1u);
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += num_ctas) {
+            const TileCoord t = tile_coord(g, tile, m_groups);
+            const CUtensorMap *m0 = swiglu ? &tmB0 : (t.map_idx == 0 ? &tmB0 : (t.map_idx == 1 ? &tmB1 : &tmB2));
+            const CUtensorMap *m1 = swiglu ? &tmB1 : m0;
+            const int brow1 = swiglu ? t.n_local : t.n_local + HALF;
+            const int kb0 = t.split * g.kb_per_split, kb1 = min(num_kb, kb0 + g.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const uint32_t s = it % (uint32_t)STAGES, ph = (it / (uint32_t)STAGES) & 1u;
+                if (!ready) ready = tc::mbar_wait(bar_empty + 8 * s, ph ^ 1u, &s_abort);
+                ok = __all_sync(0xffffffffu, ready);
+                if (!ok) break;
+                const uint32_t nx = it + 1u, ns = nx % (uint32_t)STAGES, nph = (nx / (uint32_t)STAGES) & 1u;
+                ready = tc::mbar_test(bar_empty + 8 * ns, nph ^ 1u);
+                const uint32_t sa = smem_base + s * STAGE_BYTES;
+                tc::mbar_expect_tx_elect(bar_full + 8 * s, (uint32_t)STAGE_BYTES);
+                tc::tma_load_2d_elect(sa, &tmA, kb * BK, t.m0, bar_full + 8 * s);
+                tc::tma_load_2d_elect(sa + A_BYTES, m0, kb * BK, t.n_local, bar_full + 8 * s);
+                tc::tma_load_2d_elect(sa + A_BYTES + HALF * BK * 2, m1, kb * BK, brow1, bar_full + 8 * s);
+            }
+        }
+        if (s_abort && lane == 0) {
+            // give copies already in flight a bounded chance to land before the CTA retires
+            const uint32_t first = it > (uint32_t)STAGES ? it - (uint32_t)STAGES : 0u;
+            for (uint32_t j = first; j < it; ++j) {
+                const uint32_t bar = bar_full + 8 * (j % (uint32_t)STAGES), ph = (j / (uint32_t)STAGES) & 1u;
+                for (int i = 0; i < (1 << 16) && !tc::mbar_try(bar, ph); ++i) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        const uint32_t idesc = tc::idesc_bf16_f32(BM, BN);
+        uint32_t it = 0, lt = 0;
+        bool ok = true;
+        bool ready = tc::mbar_test(bar_full, 0u);
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += num_ctas, ++lt) {
+            const uint32_t buf = lt % n_bufs, use = lt / n_bufs;
+            ok = __all_sync(0xffffffffu, tc::mbar_wait(bar_acc_empty + 8 * buf, (use & 1u) ^ 1u, &s_abort));
+            if (!ok) break;
+            tc::tc_fence_after();
+            const uint32_t d_tmem = tmem_base + buf * buf_stride;
+            const int kb0 = tile_coord(g, tile, m_groups).split * g.kb_per_split, kb1 = min(num_kb, kb0 + g.kb_per_split);
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const uint32_t s = it % (uint32_t)STAGES, ph = (it / (uint32_t)STAGES) & 1u;
+                if (!ready) ready = tc::mbar_wait(bar_full + 8 * s, ph, &s_abort);
+                ok = __all_sync(0xffffffffu, ready);
+                if (!ok) break;
+                tc::tc_fence_after();
+                const uint32_t nx = it + 1u, ns = nx % (uint32_t)STAGES, nph = (nx / (uint32_t)STAGES) & 1u;
+                ready = tc::mbar_test(bar_full + 8 * ns, nph);
+                const uint32_t sa = smem_base + s * STAGE_BYTES;
+                const uint64_t da = tc::smem_desc_sw128(sa), db = tc::smem_desc_sw128(sa + A_BYTES);
+                tc::mma_bf16_elect(d_tmem, da, db, idesc, kb != kb0 ? 1u : 0u);
+#pragma unroll
+                for (int kk = 1; kk < BK / 16; ++kk) tc::mma_bf16_elect(d_tmem, da + (uint64_t)(kk * 2), db + (uint64_t)(kk * 2), idesc, 1u);
+                tc::mma_commit_elect(bar_empty + 8 * s);          // frees the stage once these MMAs have read it
+            }
+            tc::mma_commit_elect(bar_acc_full + 8 * buf);         // accumulator complete (or abandoned)
+        }
+    } else {
+        // ---------------- epilogue: 8 warps; warp w reads TMEM lanes 32*(w%4).., the column units of parity (w-2)/4
+        const int q = warp & 3, par = (warp - 2) >> 2;
+        const uint32_t stage = smem_base + STAGES * STAGE_BYTES + kBarBytes + (uint32_t)(warp - 2) * (32 * 128);
+        uint32_t lt = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += num_ctas, ++lt) {
+            const TileCoord t = tile_coord(g, tile, m_groups);
+            const uint32_t buf = lt % n_bufs, use = lt / n_bufs;
+            ok = tc::mbar_wait(bar_acc_full + 8 * buf, use & 1u, &s_abort) && !s_abort;
+            if (!ok) break;
+            tc::tc_fence_after();
+            epilogue_tile(g, t, tmem_base + buf * buf_stride, bn_pad, stage, q, par, lane, 0, M);
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(bar_acc_empty + 8 * buf);
+        }
+    }
+
+    __syncwarp();
+    tc::tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc::tc_fence_after(); tc::tmem_dealloc(tmem_base, kTmemCols); }
+    if (threadIdx.x == 0 && s_abort && g.err) atomicExch(g.err, SFS_ERR_TIMEOUT);
+}
+
 int num_sms()
 {
     static int n = 0;
@@ -476,6 +613,40 @@ void pick_tile(int M, int K, int mode, int n_maps, int n_per_map, int pairs, int
             }
 }
 
+// Few rows: tiles of 128 x bn on single CTAs.  Per k-block a CTA streams (128 + bn) rows x 128 B at the ~40 B/clk an SM gets
+// from L2 when all SMs stream, against 2 * bn clocks of tensor-core work; 600 clocks is where the k-block time stops shrinking.
+long long model_clocks_1cta(int M, int K, int mode, int n_maps, int n_per_map, int sms, int bn, int splits)
+{
+    const long long num_kb = (K + BK - 1) / BK, kbps = (num_kb + splits - 1) / splits;
+    const long long tiles = (long long)col_tiles(mode, n_maps, n_per_map, bn) * ((num_kb + kbps - 1) / kbps);
+    const long long waves = (tiles + sms - 1) / sms;
+    const long long mma = 2LL * bn, load = (long long)(BM + bn) * 128 / 40;
+    long long kb_clk = mma > load ? mma : load;
+    if (kb_clk < 600) kb_clk = 600;
+    const long long epi = (long long)bn * 16 + 3000;
+    const long long n_out = (mode == GEMM_SWIGLU) ? n_per_map : (long long)n_maps * n_per_map;
+    const long long slab = 1500 + (long long)((double)M * (double)n_out * 1.2e-3);
+    return waves * kbps * kb_clk + epi + (splits > 1 ? slab * splits : 0);
+}
+
+void pick_tile_1cta(int M, int K, int mode, int n_maps, int n_per_map, int sms, int max_splits, int *bn_out, int *splits_out)
+{
+    const int step = (mode == GEMM_SWIGLU) ? 32 : 16;
+    long long best_cost = -1;
+    for (int bn = 256; bn >= 32; bn -= step)
+        for (int sp = 1; sp <= max_splits; ++sp) {
+            const long long cost = model_clocks_1cta(M, K, mode, n_maps, n_per_map, sms, bn, sp);
+            if (best_cost < 0 || cost < best_cost) { best_cost = cost; *bn_out = bn; *splits_out = sp; }
+        }
+}
+
+int stages_for_1cta(int bn)
+{
+    const int stage_bytes = A_BYTES + bn * BK * 2;
+    const int s = (kSmemBudget - 1024 - kBarBytes - kEpiStageBytes) / stage_bytes;
+    return s > kMaxStages ? kMaxStages : s;
+}
+
 }  // namespace
 
 int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int32_t K,
@@ -491,7 +662,10 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     SFS_REQUIRE(aligned_to(C, 16) && (ldc % 8) == 0, SFS_ERR_INVALID_ARG, "gemm: C must be 16-byte aligned, ldc a multiple of 8");
     int mb = 1, bn = 256;
     int sp_unused = 1;
-    pick_tile(M, K, mode, n_maps, n_per_map, num_sms() / 2, 1, &mb, &bn, &sp_unused);
+    // at most 128 rows: single-CTA tiles (a pair's 256-row MMA would be half padding); tune->mb = 1 or 2 forces the pair kernel
+    const bool one_cta = (M <= BM) && !(tune && (tune->mb == 1 || tune->mb == 2));
+    if (one_cta) pick_tile_1cta(M, K, mode, n_maps, n_per_map, num_sms(), 1, &bn, &sp_unused);
+    else pick_tile(M, K, mode, n_maps, n_per_map, num_sms() / 2, 1, &mb, &bn, &sp_unused);
     if (tune) {                                              // measurement overrides; invalid values are ignored
         if (tune->mb == 1 || tune->mb == 2) mb = tune->mb;
         if (tune->bn >= 32 && tune->bn <= 256 && (tune->bn % ((mode == GEMM_SWIGLU) ? 32 : 16)) == 0) bn = tune->bn;
@@ -507,12 +681,13 @@ int32_t gemm_plan_create(GemmPlan *p, const void *A, int64_t lda, int32_t M, int
     GemmArgs &g = p->args;
     g.M = M; g.N = N; g.K = K; g.mode = mode; g.out_f32 = out_f32; g.scale = scale;
     g.C = C; g.ldc = ldc; g.vt = vt; g.ldvt = ldvt; g.vt_col0 = vt_col0;
-    g.bn = bn; g.mb = mb; g.n_per_map = n_per_map;
+    g.bn = bn; g.mb = one_cta ? 1 : mb; g.n_per_map = n_per_map;
+    g.one_cta = one_cta ? 1 : 0; g.tile_rows = one_cta ? BM : mb * 2 * BM;
     g.tiles_per_map = (mode == GEMM_SWIGLU) ? 0x3FFFFFFF : (n_per_map + bn - 1) / bn;
     g.n_col_tiles = col_tiles(mode, n_maps, n_per_map, bn);
-    g.stages = stages_for(mb, bn);
+    g.stages = one_cta ? stages_for_1cta(bn) : stages_for(mb, bn);
     if (tune && tune->stages >= 1 && tune->stages <= g.stages) g.stages = tune->stages;
-    g.acc_bufs = (mb * ((bn + 31) & ~31) <= 256) ? 2 : 1;
+    g.acc_bufs = (g.mb * ((bn + 31) & ~31) <= 256) ? 2 : 1;
     g.splits = 1; g.kb_per_split = (K + BK - 1) / BK; g.split_stride = 0;
     p->A = A; p->lda = lda; p->ldb = ldb;
     for (int i = 0; i < 3; ++i) p->Bs[i] = Bs[i < n_maps ? i : 0];
@@ -525,7 +700,9 @@ int32_t gemm_plan_enable_split(GemmPlan *p, float *ws, int32_t max_splits, const
     const bool f32_out = g.mode == GEMM_RESIDUAL_F32 || (g.mode == GEMM_STORE && g.out_f32 && g.vt == nullptr);
     if (!f32_out || ws == nullptr || max_splits < 2) return SFS_OK;
     int mb = g.mb, bn = g.bn, sp = 1;
-    pick_tile(g.M, g.K, g.mode, p->n_maps, p->n_per_map, num_sms() / 2, max_splits, &mb, &bn, &sp);
+    const bool one_cta = g.one_cta != 0;
+    if (one_cta) pick_tile_1cta(g.M, g.K, g.mode, p->n_maps, p->n_per_map, num_sms(), max_splits, &bn, &sp);
+    else pick_tile(g.M, g.K, g.mode, p->n_maps, p->n_per_map, num_sms() / 2, max_splits, &mb, &bn, &sp);
     if (tune) {
         if (tune->mb == 1 || tune->mb == 2) mb = tune->mb;
         if (tune->bn >= 32 && tune->bn <= 256 && (tune->bn % 16) == 0) bn = tune->bn;
@@ -534,7 +711,7 @@ int32_t gemm_plan_enable_split(GemmPlan *p, float *ws, int32_t max_splits, const
     if (sp <= 1 && !tune) return SFS_OK;
     // rebuild the plan at the new tile shape, then cut K
     GemmPlan q;
-    GemmTune t2 = {mb, bn, tune ? tune->stages : 0, 0};
+    GemmTune t2 = {one_cta ? 0 : mb, bn, tune ? tune->stages : 0, 0};
     int32_t rc = gemm_plan_create(&q, p->A, p->lda, g.M, g.K, p->Bs, p->n_maps, p->n_per_map, p->ldb, g.mode, g.C, g.ldc, g.out_f32,
                                   g.scale, g.vt, g.ldvt, g.vt_col0, &t2);
     if (rc != SFS_OK) return rc;
@@ -563,6 +740,21 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
     }
     GemmArgs g = p.args;
     g.d_m = d_m; g.err = err; g.d_active = d_active;
+    if (g.one_cta) {
+        static bool configured1[kMaxDevices] = {};
+        bool &done1 = configured1[current_device_slot()];
+        if (!done1) {
+            SFS_CUDA(cudaFuncSetAttribute(gemm_kernel_1cta, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+            done1 = true;
+        }
+        size_t smem1 = (size_t)g.stages * (A_BYTES + g.bn * BK * 2) + kBarBytes + kEpiStageBytes + 1024;
+        if (smem1 < 120 * 1024) smem1 = 120 * 1024;            // one CTA per SM: all 512 tensor-memory columns are its own
+        const long long tiles1 = (long long)((g.M + BM - 1) / BM) * g.n_col_tiles * g.splits;
+        const int sms = num_sms();
+        gemm_kernel_1cta<<<(unsigned)(tiles1 < sms ? tiles1 : sms), kGemmThreads, smem1, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
+        SFS_LAUNCH_CHECK();
+        return SFS_OK;
+    }
     size_t smem = (size_t)g.stages * (g.mb * A_BYTES + (g.bn / 2) * BK * 2) + kBarBytes + kEpiStageBytes + 1024;
     if (smem < 120 * 1024) smem = 120 * 1024;
     const long long tiles = (long long)((g.M + g.mb * 2 * BM - 1) / (g.mb * 2 * BM)) * g.n_col_tiles * g.splits;

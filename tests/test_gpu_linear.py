@@ -55,3 +55,14 @@ def test_linear_few_wide_tiles(M, N, K, out_dtype):
             # one bf16 rounding (half an ulp: up to 2^-8 relative) of an fp32 sum of K products whose own error grows with K
             rel = np.abs(got - ref) / np.maximum(np.abs(ref), 1.0)
             assert rel.max() <= 2.0 ** -8 + 1e-7 * K
+
+
+@pytest.mark.parametrize("M,N,K,out_dtype", [(128, 12288, 4096, 0), (128, 4096, 12288, 1), (77, 4096, 4096, 1), (128, 126464, 512, 0), (5, 3000, 1024, 0)])
+def test_linear_few_rows(M, N, K, out_dtype):
+    """At most 128 rows: the single-CTA tiles (weights streamed through every SM), at the widths of the cached partial steps."""
+    got, ref = run(M, N, K, out_dtype, seed=11)
+    if out_dtype:
+        assert np.abs(got - ref).max() <= 1e-3 * np.abs(ref).max()
+    else:
+        rel = np.abs(got - ref) / np.maximum(np.abs(ref), 1.0)
+        assert rel.max() <= 2.0 ** -8 + 1e-7 * K
