@@ -76,7 +76,7 @@ static int32_t dev_alloc(sfs_session *s, T **out, size_t count, bool zero)
 static int32_t step_row_stats(sfs_session *s, const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld,
                               const int32_t *d_n_rows, int32_t max_rows, const int32_t *d_rows, const uint8_t *d_mask,
                               int32_t B, int32_t S, int32_t P, const sfs_state *d_state, const sfs_params &params, bool *two_pass,
-                              cudaStream_t st)
+                              cudaStream_t st, const float4 *lm_stats = nullptr, int32_t lm_stats_ld = 0)
 {
     int32_t *err = device_status_word();
     *two_pass = row_stats_two_pass_applies(d_logits, logits_dtype, vocab, ld);
@@ -88,6 +88,8 @@ static int32_t step_row_stats(sfs_session *s, const void *d_logits, int32_t logi
     rf.pos_lo = s->pos_lo; rf.pos_hi = s->pos_hi; rf.pos_sq = s->pos_sq; rf.pos_arg = s->pos_arg;
     rf.slice_partials = s->slice_partials; rf.row_tickets = s->row_tickets;
     rf.pos_row = s->pos_row; rf.pos_max = s->pos_max; rf.refine_list = s->refine_list; rf.refine_count = s->refine_count;
+    if (lm_stats != nullptr)       // the LM head's epilogue has taken the first pass: the logits are read only for the listed rows
+        return launch_row_stats_from_partials(lm_stats, lm_stats_ld, lm_stats_ld, d_logits, vocab, ld, d_n_rows, max_rows, d_rows, rf, err, st);
     return launch_row_stats_two_pass(d_logits, vocab, ld, d_n_rows, max_rows, d_rows, rf, err, st);
 }
 
@@ -726,6 +728,23 @@ int32_t sfs_generate_begin(sfs_session *s, const int32_t *d_prompt, int32_t B, i
         rc = gemm_plan_create(&s->lm_plan, s->hfin, c.d_model, B * gen_len, c.d_model, lm, 1, c.vocab, c.d_model, GEMM_STORE,
                               s->logits, c.vocab, 0, c.logit_scale, nullptr, 0, 0, nullptr);
         if (rc != SFS_OK) return rc;
+        // Long bf16 rows: the LM head takes the first pass of the row statistics in its epilogue (one record per row,
+        // column tile and epilogue-warp parity), so the selection step never streams the logits back from memory.
+        // (tiles of at least 128 columns: then both epilogue-warp parities own columns of every 256-row block)
+        if (row_stats_two_pass_applies(s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab) && s->lm_plan.args.splits == 1 && s->lm_plan.args.bn >= 128) {
+            const int parts = 2 * s->lm_plan.args.n_col_tiles;
+            const size_t need = (size_t)B * gen_len * parts;
+            if (s->lm_stats_cap < need) {
+                SFS_CUDA(cudaStreamSynchronize(st));
+                if (s->lm_stats) {
+                    for (auto it = s->owned.begin(); it != s->owned.end(); ++it) if (*it == (void *)s->lm_stats) { s->owned.erase(it); break; }
+                    cudaFree(s->lm_stats); s->lm_stats = nullptr; s->lm_stats_cap = 0;
+                }
+                if ((rc = dev_alloc(s, &s->lm_stats, need, true)) != SFS_OK) return rc;
+                s->lm_stats_cap = need;
+            }
+            s->lm_plan.args.stats = s->lm_stats; s->lm_plan.args.stats_ld = parts;
+        }
     }
     generate_init_kernel<<<64, 256, 0, st>>>(d_prompt, s->tokens, s->mask, s->rows[0], s->ctrl, s->host_active_dev, s->pos_sq,
                                              B, P, gen_len, s->model->cfg.mask_id);
@@ -769,7 +788,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         bool two_pass = false;
         if ((rc = timed_launch(s, SFS_K_ROW_STATS, st, [&] {
                  return step_row_stats(s, s->logits, SFS_LOGITS_BF16, c.vocab, c.vocab, n_rows, B * L, rows, s->mask, B, S, P, s->state,
-                                       s->gen_params, &two_pass, st); })) != SFS_OK) return rc;
+                                       s->gen_params, &two_pass, st, s->lm_plan.args.stats, s->lm_plan.args.stats_ld); })) != SFS_OK) return rc;
         SelectArgs a{};
         a.pos_lo = two_pass ? s->pos_lo : nullptr;
         a.tokens = s->tokens; a.mask = s->mask; a.B = B; a.S = S; a.P = P; a.L = L;

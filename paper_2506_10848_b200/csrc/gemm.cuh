@@ -29,6 +29,11 @@ struct GemmArgs {
     int splits, kb_per_split;        // split-K: the k-blocks are cut into `splits` ranges, range s writes slab s of C
     long long split_stride;          // elements between slabs
     int acc_bufs;            // accumulator buffers in tensor memory (2 when they fit: epilogue overlaps the next tile)
+    // Optional (GEMM_STORE, bf16 output, no split): row statistics of the stored values, taken in the epilogue.  Per output
+    // row, column tile and epilogue-warp parity one record (maximum, reference, sum of 2^((x - reference) log2 e), first
+    // position of the maximum as int bits) at stats[row * stats_ld + 2 * column_tile + parity]: the first pass of the
+    // selection step's row statistics, fused into the LM head (the logits are not read back for it).
+    float4 *stats; int stats_ld;
     int32_t *err;            // device status word, set to SFS_ERR_TIMEOUT if a bounded wait gives up
     const int32_t *d_active; // optional: the kernel does nothing when *d_active == 0
 };

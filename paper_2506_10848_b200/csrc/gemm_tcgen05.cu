@@ -160,6 +160,7 @@ __device__ __forceinline__ void flush_unit(const GemmArgs &g, long long slab, ui
 // A unit may reach past the tile's valid columns: those accumulator columns exist (inside the 256-column buffer) and
 // are never stored.  The tensor-memory loads of the next piece are issued as soon as the current piece has been
 // converted, so their latency hides behind the parking and the stores of the current one.
+template <bool STATS>
 __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord &t, uint32_t tmem_acc, uint32_t bn_pad, uint32_t stage,
                                               int q, int par, int lane, int rank, int M)
 {
@@ -182,6 +183,16 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
             tc::tmem_ld32(piece_addr(0), x0);
             if (swiglu) tc::tmem_ld32(piece_addr(0) + HALF, x1);
         }
+        // fused row statistics (LM head): this lane's row of the current 256-row block
+        const bool stats_on = STATS && (g.stats != nullptr) && !swiglu;
+        float st_mx = -INFINITY, st_ref = 0.f, st_nref = 0.f, st_sum = 0.f;
+        int st_arg = 0x7FFFFFFF, st_b = -1;
+        const int n_tile = (t.ncol0 / g.bn);                             // one weight matrix: column tile index
+        auto stats_flush = [&]() {
+            if (st_b < 0) return;
+            const int grow = grow_q + st_b * 2 * BM + lane;
+            if (grow < M) g.stats[(long long)grow * g.stats_ld + 2 * n_tile + par] = make_float4(st_mx, st_ref, st_sum, __int_as_float(st_arg));
+        };
         for (int pc = 0; pc < n_pieces; ++pc) {
             uint32_t o[16];
             tc::tmem_ld_wait32(x0);
@@ -199,6 +210,42 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
                 tc::tmem_ld32(piece_addr(pc + 1), x0);
                 if (swiglu) tc::tmem_ld32(piece_addr(pc + 1) + HALF, x1);
             }
+            if (stats_on) {
+                // statistics of the ROUNDED values, as a reader of the stored logits would see them
+                const int u = par + 2 * (pc >> 1), b = u / upb, col0 = t.ncol0 + 64 * (u - b * upb) + 32 * (pc & 1);
+                if (b != st_b) { stats_flush(); st_b = b; st_mx = -INFINITY; st_sum = 0.f; st_arg = 0x7FFFFFFF; st_ref = 0.f; st_nref = 0.f; }
+                const int nvalid = min(32, lim - col0);                  // columns of this piece inside the matrix (warp-uniform)
+                float pm = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float lo = __uint_as_float(o[j] << 16), hi = __uint_as_float(o[j] & 0xFFFF0000u);
+                    if (2 * j < nvalid) pm = fmaxf(pm, lo);
+                    if (2 * j + 1 < nvalid) pm = fmaxf(pm, hi);
+                }
+                if (st_mx == -INFINITY && st_sum == 0.f) {               // first piece of this row: it gives the reference
+                    st_ref = (fabsf(pm) <= 3.0e38f) ? pm : 0.f;
+                    st_nref = -st_ref * 1.4426950408889634f;
+                }
+                if (pm > st_mx) {                                        // strict: the first position of the maximum
+                    st_mx = pm;
+#pragma unroll
+                    for (int j = 15; j >= 0; --j) {
+                        const float lo = __uint_as_float(o[j] << 16), hi = __uint_as_float(o[j] & 0xFFFF0000u);
+                        if (2 * j + 1 < nvalid && hi == pm) st_arg = col0 + 2 * j + 1;
+                        if (2 * j < nvalid && lo == pm) st_arg = col0 + 2 * j;
+                    }
+                }
+                float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float lo = __uint_as_float(o[j] << 16), hi = __uint_as_float(o[j] & 0xFFFF0000u);
+                    const float e0 = tc::ex2_approx(__fmaf_rn(lo, 1.4426950408889634f, st_nref));
+                    const float e1 = tc::ex2_approx(__fmaf_rn(hi, 1.4426950408889634f, st_nref));
+                    s0 += (2 * j < nvalid) ? e0 : 0.f;
+                    s1 += (2 * j + 1 < nvalid) ? e1 : 0.f;
+                }
+                st_sum += s0 + s1;
+            }
             park16(stage, lane, 4 * (pc & 1), o);
             if (pc & 1) {
                 const int u = par + 2 * (pc >> 1), b = u / upb, c = 64 * (u - b * upb);
@@ -207,6 +254,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
                 __syncwarp();
             }
         }
+        if (stats_on) stats_flush();
     } else if (g.vt != nullptr && t.ncol0 >= g.vt_col0) {
         // ---- V columns of the QKV projection go out transposed: the 32 lanes hold 32 consecutive tokens of a feature
         const int upb = (t.ncols + 31) / 32;
@@ -259,6 +307,7 @@ __device__ __forceinline__ void epilogue_tile(const GemmArgs &g, const TileCoord
     }
 }
 
+template <bool STATS>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
@@ -399,7 +448,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             ok = tc::mbar_wait(bar_acc_full + 8 * buf, use & 1u, &s_abort) && !s_abort;
             if (!ok) break;
             tc::tc_fence_after();
-            epilogue_tile(g, t, tmem_base + buf * buf_stride, bn_pad, stage, q, par, lane, (int)rank, M);
+            epilogue_tile<STATS>(g, t, tmem_base + buf * buf_stride, bn_pad, stage, q, par, lane, (int)rank, M);
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive_cluster(lead_acc_empty + 8 * buf);
@@ -420,6 +469,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
 // tcgen05.mma.cta_group::1 (M = 128, N = BN), loading the 128 activation rows and BN weight rows of every k-block itself (the
 // weight rows as two boxes of BN / 2, SwiGLU: gate rows then up rows, so the accumulator layout and the epilogue are those
 // of the pair kernel); BN is chosen so that the tiles fill the SMs in whole waves.  Same warp roles, ring and bounded waits.
+template <bool STATS>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel_1cta(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
@@ -537,7 +587,7 @@ gemm_kernel_1cta(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ok = tc::mbar_wait(bar_acc_full + 8 * buf, use & 1u, &s_abort) && !s_abort;
             if (!ok) break;
             tc::tc_fence_after();
-            epilogue_tile(g, t, tmem_base + buf * buf_stride, bn_pad, stage, q, par, lane, 0, M);
+            epilogue_tile<STATS>(g, t, tmem_base + buf * buf_stride, bn_pad, stage, q, par, lane, 0, M);
             tc::tc_fence_before();
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(bar_acc_empty + 8 * buf);
@@ -735,7 +785,8 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
     static bool configured[kMaxDevices] = {};
     bool &done = configured[current_device_slot()];
     if (!done) {
-        SFS_CUDA(cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        SFS_CUDA(cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+        SFS_CUDA(cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
         done = true;
     }
     GemmArgs g = p.args;
@@ -744,14 +795,17 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
         static bool configured1[kMaxDevices] = {};
         bool &done1 = configured1[current_device_slot()];
         if (!done1) {
-            SFS_CUDA(cudaFuncSetAttribute(gemm_kernel_1cta, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+            SFS_CUDA(cudaFuncSetAttribute(gemm_kernel_1cta<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
+            SFS_CUDA(cudaFuncSetAttribute(gemm_kernel_1cta<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBudget));
             done1 = true;
         }
         size_t smem1 = (size_t)g.stages * (A_BYTES + g.bn * BK * 2) + kBarBytes + kEpiStageBytes + 1024;
         if (smem1 < 120 * 1024) smem1 = 120 * 1024;            // one CTA per SM: all 512 tensor-memory columns are its own
         const long long tiles1 = (long long)((g.M + BM - 1) / BM) * g.n_col_tiles * g.splits;
         const int sms = num_sms();
-        gemm_kernel_1cta<<<(unsigned)(tiles1 < sms ? tiles1 : sms), kGemmThreads, smem1, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
+        const unsigned grid1 = (unsigned)(tiles1 < sms ? tiles1 : sms);
+        if (g.stats) gemm_kernel_1cta<true><<<grid1, kGemmThreads, smem1, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
+        else gemm_kernel_1cta<false><<<grid1, kGemmThreads, smem1, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
         SFS_LAUNCH_CHECK();
         return SFS_OK;
     }
@@ -760,7 +814,8 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
     const long long tiles = (long long)((g.M + g.mb * 2 * BM - 1) / (g.mb * 2 * BM)) * g.n_col_tiles * g.splits;
     const int pairs = num_sms() / 2;
     dim3 grid((unsigned)(2 * (tiles < pairs ? tiles : pairs)), 1, 1);
-    gemm_kernel<<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
+    if (g.stats) gemm_kernel<true><<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
+    else gemm_kernel<false><<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
     SFS_LAUNCH_CHECK();
     return SFS_OK;
 }

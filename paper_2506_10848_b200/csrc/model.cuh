@@ -56,6 +56,7 @@ struct sfs_session {
     std::vector<LayerPlans> layer_plans;
     sfs::AttnPlan attn_plan;
     sfs::GemmPlan lm_plan;
+    float4 *lm_stats = nullptr; size_t lm_stats_cap = 0;     // row-statistics records the LM head's epilogue leaves (fused first pass)
     // what the next RMSNorm must fold into x: n slabs `pending_stride` floats apart (split-K partials or a cached increment)
     const float *pending_ptr = nullptr; int pending_n = 0; long long pending_stride = 0;
     // feature cache (dLLM-Cache-style), allocated by sfs_cache_enable

@@ -472,6 +472,64 @@ struct BoundsOut {
     int32_t *tickets;                                       // scratch [max_rows], zero between launches
 };
 
+// the enclosure of the canonical S_q from the approximate sum `tot` (relative to the row maximum m), and the scattered outputs
+__device__ __forceinline__ void write_enclosure(const BoundsOut &out, int row, float tot, int arg, float m, bool open, int vocab)
+{
+    if (arg == 0x7FFFFFFF) arg = 0;
+    const double Sd = (double)tot * (double)(1u << SFS_CONF_QBITS);
+    const double dlo = Sd * (1.0 - kEps) - (double)vocab - 1.0, dhi = Sd * (1.0 + kEps) + 1.0;
+    const unsigned long long floor_q = 1ull << SFS_CONF_QBITS;     // the maximum alone contributes 2^28
+    unsigned long long lo = dlo > (double)floor_q ? (unsigned long long)dlo : floor_q;
+    unsigned long long hi = (unsigned long long)dhi + 1ull;
+    if (open || !(tot >= 0.999f) || !(tot <= 3.0e38f)) { lo = 1ull; hi = ~0ull >> 1; }
+    if (out.lo) out.lo[row] = lo;
+    if (out.hi) out.hi[row] = hi;
+    if (out.argmax) out.argmax[row] = arg;
+    if (out.rows && out.pos_lo) {
+        const int p = out.rows[row];
+        if ((unsigned)p < (unsigned)out.n_positions) {
+            out.pos_lo[p] = lo; out.pos_hi[p] = hi; out.pos_arg[p] = arg; out.pos_row[p] = row; out.pos_max[p] = m;
+        } else if (out.err) {
+            atomicExch(out.err, SFS_ERR_INVALID_ARG);
+        }
+    }
+}
+
+// Pass 1 when the LM head has already taken the statistics in its epilogue: per row, n_parts records (maximum, reference,
+// sum of 2^((x - reference) log2 e), first position of the maximum) are combined exactly like the slices of the streaming
+// kernel — one warp per row, the lanes' shares added in a fixed order — into the row's argmax and enclosure.  The logits are
+// not read.
+__global__ void __launch_bounds__(128)
+combine_partials_kernel(const float4 *__restrict__ stats, int stats_ld, int n_parts, const int32_t *__restrict__ n_rows_ptr, int max_rows,
+                        int vocab, BoundsOut out)
+{
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    const int n_rows = n_rows_ptr ? min(*n_rows_ptr, max_rows) : max_rows;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && out.list_count) *out.list_count = 0;
+    if (row >= n_rows) return;
+    const float4 *ps = stats + (long long)row * stats_ld;
+    float m = -INFINITY;
+    for (int q = lane; q < n_parts; q += 32) m = fmaxf(m, __ldg(&ps[q]).x);
+    m = warp_max(m);
+    const float nm = __fmul_rn(-m, kLog2e);
+    int arg = 0x7FFFFFFF;
+    float tot = 0.f;
+    int open = 0;
+    for (int q = lane; q < n_parts; q += 32) {
+        const float4 r = __ldg(&ps[q]);
+        if (r.x == m) arg = min(arg, __float_as_int(r.w));
+        if (r.z != 0.f) {
+            const float shift = __fmaf_rn(r.y, kLog2e, nm);
+            if (!(shift >= -100.f) || !(shift <= 100.f)) open = 1;
+            tot += r.z * ex2_fast(shift);
+        }
+    }
+    tot = warp_sum(tot);
+    arg = warp_min_i32(arg);
+    open = warp_max_i32(open);
+    if (lane == 0) write_enclosure(out, row, tot, arg, m, open != 0, vocab);
+}
+
 __device__ __forceinline__ uint32_t chunk_max2(const uint4 &v) {
     __nv_bfloat162 m = __hmax2(__hmax2(as_bf162(v.x), as_bf162(v.y)), __hmax2(as_bf162(v.z), as_bf162(v.w)));
     return *reinterpret_cast<uint32_t *>(&m);
@@ -619,24 +677,7 @@ rowstats_bounds_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int 
             tot += ps[q].z * ex2_fast(shift);
         }
     }
-    if (arg == 0x7FFFFFFF) arg = 0;
-    const double Sd = (double)tot * (double)(1u << SFS_CONF_QBITS);
-    const double dlo = Sd * (1.0 - kEps) - (double)vocab - 1.0, dhi = Sd * (1.0 + kEps) + 1.0;
-    const unsigned long long floor_q = 1ull << SFS_CONF_QBITS;     // the maximum alone contributes 2^28
-    unsigned long long lo = dlo > (double)floor_q ? (unsigned long long)dlo : floor_q;
-    unsigned long long hi = (unsigned long long)dhi + 1ull;
-    if (open || !(tot >= 0.999f) || !(tot <= 3.0e38f)) { lo = 1ull; hi = ~0ull >> 1; }
-    if (out.lo) out.lo[row] = lo;
-    if (out.hi) out.hi[row] = hi;
-    if (out.argmax) out.argmax[row] = arg;
-    if (out.rows && out.pos_lo) {
-        const int p = out.rows[row];
-        if ((unsigned)p < (unsigned)out.n_positions) {
-            out.pos_lo[p] = lo; out.pos_hi[p] = hi; out.pos_arg[p] = arg; out.pos_row[p] = row; out.pos_max[p] = m;
-        } else if (out.err) {
-            atomicExch(out.err, SFS_ERR_INVALID_ARG);
-        }
-    }
+    write_enclosure(out, row, tot, arg, m, open, vocab);
 }
 
 // Pass 2 of the two-pass form, second half: the canonical S_q of the listed rows.  Pass 1 has left the exact row maximum, so one
@@ -909,6 +950,25 @@ int32_t launch_row_stats_two_pass(const void *d_logits, int32_t vocab, int64_t l
     if (rc != SFS_OK) return rc;
     refine_decide_kernel<<<rf.B, kDecideThreads, 0, stream>>>(rf);
     SFS_LAUNCH_CHECK();
+    const int items = max_rows * kListParts, cap = 2 * num_sms_rowstats();
+    rowstats_list_bf16<<<items < cap ? items : cap, kListThreads, 0, stream>>>(lp, ld / 8, vocab / 8, d_rows, rf.refine_list, rf.refine_count,
+                                                                              rf.pos_max, rf.pos_sq, rf.B * rf.S);
+    SFS_LAUNCH_CHECK();
+    return SFS_OK;
+}
+
+int32_t launch_row_stats_from_partials(const void *stats, int32_t stats_ld, int32_t n_parts, const void *d_logits, int32_t vocab, int64_t ld,
+                                       const int32_t *d_n_rows, int32_t max_rows, const int32_t *d_rows, const RefineArgs &rf, int32_t *d_err,
+                                       cudaStream_t stream)
+{
+    if (max_rows <= 0) return SFS_OK;
+    BoundsOut bo{d_rows, nullptr, nullptr, nullptr, rf.pos_lo, rf.pos_hi, rf.pos_arg, rf.pos_row, rf.pos_max, rf.refine_count, rf.B * rf.S, d_err,
+                 nullptr, nullptr};
+    combine_partials_kernel<<<(max_rows + 3) / 4, 128, 0, stream>>>(reinterpret_cast<const float4 *>(stats), stats_ld, n_parts, d_n_rows, max_rows, vocab, bo);
+    SFS_LAUNCH_CHECK();
+    refine_decide_kernel<<<rf.B, kDecideThreads, 0, stream>>>(rf);
+    SFS_LAUNCH_CHECK();
+    const uint4 *lp = reinterpret_cast<const uint4 *>(d_logits);
     const int items = max_rows * kListParts, cap = 2 * num_sms_rowstats();
     rowstats_list_bf16<<<items < cap ? items : cap, kListThreads, 0, stream>>>(lp, ld / 8, vocab / 8, d_rows, rf.refine_list, rf.refine_count,
                                                                               rf.pos_max, rf.pos_sq, rf.B * rf.S);

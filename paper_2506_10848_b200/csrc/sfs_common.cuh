@@ -158,6 +158,10 @@ constexpr int kRowStatsSlices = 8;
 bool row_stats_two_pass_applies(const void *d_logits, int32_t logits_dtype, int32_t vocab, int64_t ld);
 int32_t launch_row_stats_two_pass(const void *d_logits, int32_t vocab, int64_t ld, const int32_t *d_n_rows, int32_t max_rows,
                                   const int32_t *d_rows, const RefineArgs &rf, int32_t *d_err, cudaStream_t stream);
+// the same with pass 1 already taken by the LM head's epilogue: `stats` holds n_parts records per row (stats_ld apart)
+int32_t launch_row_stats_from_partials(const void *stats, int32_t stats_ld, int32_t n_parts, const void *d_logits, int32_t vocab, int64_t ld,
+                                       const int32_t *d_n_rows, int32_t max_rows, const int32_t *d_rows, const RefineArgs &rf, int32_t *d_err,
+                                       cudaStream_t stream);
 // pass 1 alone, dense outputs by logits row (for tests): d_lo / d_hi enclose the canonical S_q
 int32_t launch_row_stats_bounds(const void *d_logits, int32_t vocab, int64_t ld, const int32_t *d_n_rows, int32_t max_rows,
                                 unsigned long long *d_lo, unsigned long long *d_hi, int32_t *d_argmax, int32_t *d_err, cudaStream_t stream);
