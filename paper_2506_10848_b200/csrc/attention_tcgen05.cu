@@ -34,6 +34,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     constexpr int P_BYTES = QT * KT * 2;
     constexpr uint32_t TMEM_COLS = 512;                  // S (two buffers of 128 columns) and O (DH columns)
 
+    pdl_wait();                                          // the kernel before this one in the stream has completed
+    pdl_trigger();
     if (a.d_active && *a.d_active == 0) return;          // nothing left to decode: uniform early exit
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -304,8 +306,7 @@ int32_t launch_dh(const AttnPlan &p, int kq, const int32_t *d_active, int32_t *e
     a.err = err; a.d_active = d_active;
     if (kq > 0) a.kq = kq;
     dim3 grid((unsigned)((a.kq + QT - 1) / QT), (unsigned)a.n_heads, (unsigned)a.B);
-    attention_kernel<DH><<<grid, kAttnThreads, smem, stream>>>(p.tmQ, p.tmK, p.tmVt, a);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(attention_kernel<DH>, grid, dim3(kAttnThreads), smem, stream, p.tmQ, p.tmK, p.tmVt, a));
     return SFS_OK;
 }
 

@@ -36,6 +36,8 @@ rmsnorm_kernel(float *__restrict__ x, const float *__restrict__ partial, int n_p
                const __nv_bfloat16 *__restrict__ gain, __nv_bfloat16 *__restrict__ h,
                const int32_t *__restrict__ rows, const int32_t *__restrict__ n_rows_ptr, int max_rows, int d, float eps)
 {
+    pdl_wait();
+    pdl_trigger();
     const int n_rows = n_rows_ptr ? min(*n_rows_ptr, max_rows) : max_rows;
     __shared__ float s_part[kNormThreads / 32];
     const int chunks = d / 4;
@@ -117,6 +119,8 @@ __global__ void rope_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int T,
                             const float2 *__restrict__ table, const int32_t *__restrict__ rows)
 {
     // one thread handles 8 consecutive j of one (token, q-or-k, head)
+    pdl_wait();
+    pdl_trigger();
     const int half = dh / 2, groups = half / 8;
     const unsigned idx = blockIdx.x * blockDim.x + threadIdx.x;   // the launcher checks that the item count fits 31 bits
     const unsigned total = (unsigned)T * 2u * (unsigned)n_heads * (unsigned)groups;
@@ -165,9 +169,8 @@ int32_t launch_rmsnorm(float *x, const float *partial, int n_partial, long long 
     if (max_rows <= 0) return SFS_OK;
     const int grid = max_rows < 148 * 16 ? max_rows : 148 * 16;
     if (partial == nullptr) n_partial = 0;
-    rmsnorm_kernel<<<grid, kNormThreads, 0, s>>>(x, partial ? partial : x, n_partial, partial_stride, reinterpret_cast<const __nv_bfloat16 *>(gain),
-                                                 reinterpret_cast<__nv_bfloat16 *>(h), rows, n_rows, max_rows, d, eps);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(rmsnorm_kernel, dim3(grid), dim3(kNormThreads), 0, s, x, partial ? partial : x, n_partial, partial_stride,
+                        reinterpret_cast<const __nv_bfloat16 *>(gain), reinterpret_cast<__nv_bfloat16 *>(h), rows, n_rows, max_rows, d, eps));
     return SFS_OK;
 }
 
@@ -183,8 +186,8 @@ int32_t launch_rope(void *qk, int64_t ld, int T, int S, int n_heads, int head_di
 {
     const long long total = (long long)T * 2 * n_heads * (head_dim / 16);
     SFS_REQUIRE(total < (1LL << 31), SFS_ERR_INVALID_ARG, "rope: %lld items do not fit a 32-bit index", total);
-    rope_kernel<<<(unsigned)((total + 255) / 256), 256, 0, s>>>(reinterpret_cast<__nv_bfloat16 *>(qk), ld, T, S, n_heads, head_dim, table, rows);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(rope_kernel, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, s, reinterpret_cast<__nv_bfloat16 *>(qk), (long long)ld, T, S,
+                        n_heads, head_dim, table, rows));
     return SFS_OK;
 }
 

@@ -312,6 +312,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
 {
+    pdl_wait();                                             // the kernel before this one in the stream has completed
+    pdl_trigger();
     // the exits below are uniform over the pair (same values in both CTAs), before any barrier or allocation
     if (g.d_active && *g.d_active == 0) return;             // nothing left to decode
     const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
@@ -814,9 +816,8 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
     const long long tiles = (long long)((g.M + g.mb * 2 * BM - 1) / (g.mb * 2 * BM)) * g.n_col_tiles * g.splits;
     const int pairs = num_sms() / 2;
     dim3 grid((unsigned)(2 * (tiles < pairs ? tiles : pairs)), 1, 1);
-    if (g.stats) gemm_kernel<true><<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
-    else gemm_kernel<false><<<grid, kGemmThreads, smem, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
-    SFS_LAUNCH_CHECK();
+    if (g.stats) SFS_CUDA(launch_pdl(gemm_kernel<true>, grid, dim3(kGemmThreads), smem, stream, p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g));
+    else SFS_CUDA(launch_pdl(gemm_kernel<false>, grid, dim3(kGemmThreads), smem, stream, p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g));
     return SFS_OK;
 }
 

@@ -47,6 +47,26 @@ static inline int current_device_slot()
 int32_t *device_status_word();
 int32_t *device_status_word_if_any();
 
+// ---- programmatic dependent launch -----------------------------------------------------------------------
+// A kernel launched with launch_pdl may start (be scheduled, run its prologue) while the kernel before it in the stream is
+// still running; it calls pdl_wait() before its first access to global memory, which returns once that kernel has completed
+// and its writes are visible.  pdl_trigger() tells the runtime that the kernels after this one may be scheduled.
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // ---- device helpers ---------------------------------------------------------------------------------
 #ifdef __CUDACC__
 __device__ __forceinline__ float bf16_bits_to_f32(uint32_t h16) { return __uint_as_float(h16 << 16); }
