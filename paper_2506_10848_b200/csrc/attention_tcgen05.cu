@@ -34,9 +34,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     constexpr int P_BYTES = QT * KT * 2;
     constexpr uint32_t TMEM_COLS = 512;                  // S (two buffers of 128 columns) and O (DH columns)
 
-    pdl_wait();                                          // the kernel before this one in the stream has completed
-    pdl_trigger();
-    if (a.d_active && *a.d_active == 0) return;          // nothing left to decode: uniform early exit
+    pdl_trigger();                                       // (may run beside the end of the kernel before it: see pdl_wait below)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = smem, *sK = smem + Q_BYTES, *sV = sK + KV_STAGES * K_BYTES, *sP = sV + KV_STAGES * V_BYTES;
@@ -73,6 +71,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t *>(tmem_slot);
     const uint32_t tmem_S = tmem_base, tmem_O = tmem_base + 2 * KT;
 
+    pdl_wait();                                          // the kernel before this one has completed: global memory from here on
+    const bool live = !(a.d_active && *a.d_active == 0); // nothing left to decode: straight to the teardown (uniform)
+    if (live) {
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer: Q once, then K tiles and V^T tiles through their own rings (a K stage is free
@@ -284,6 +285,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             }
         }
     }
+    }   // live
 
     tc::tc_fence_before();
     __syncthreads();

@@ -312,16 +312,13 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
             const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
 {
-    pdl_wait();                                             // the kernel before this one in the stream has completed
+    // This kernel may have been scheduled while the one before it in the stream still runs (programmatic dependent launch):
+    // everything up to pdl_wait() touches only this CTA's shared and tensor memory.
     pdl_trigger();
-    // the exits below are uniform over the pair (same values in both CTAs), before any barrier or allocation
-    if (g.d_active && *g.d_active == 0) return;             // nothing left to decode
-    const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
     const int MB = g.mb;
-    const int m_groups = (M + MB * 2 * BM - 1) / (MB * 2 * BM);
-    const int num_tiles = m_groups * g.n_col_tiles * g.splits;
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    if (pair >= num_tiles) return;
+    // uniform over the pair, before any barrier or allocation: pairs beyond the tiles of even the largest row count
+    if (pair >= ((g.M + MB * 2 * BM - 1) / (MB * 2 * BM)) * g.n_col_tiles * g.splits) return;
 
     const int BN = g.bn, STAGES = g.stages, HALF = BN >> 1;
     const int STAGE_BYTES = MB * A_BYTES + HALF * BK * 2;   // per CTA: MB blocks of 128 A rows, half of the weight rows
@@ -356,6 +353,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t bn_pad = (uint32_t)((BN + 31) & ~31);
     const uint32_t n_bufs = (uint32_t)g.acc_bufs, buf_stride = 256;     // two buffers only when MB * bn_pad <= 256
     const bool swiglu = (g.mode == GEMM_SWIGLU);
+
+    pdl_wait();                                             // the kernel before this one has completed: global memory from here on
+    // nothing left to decode, or fewer rows than planned: the loops below find no tile (same values in both CTAs of the pair)
+    const bool live = !(g.d_active && *g.d_active == 0);
+    const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
+    const int m_groups = (M + MB * 2 * BM - 1) / (MB * 2 * BM);
+    const int num_tiles = live ? m_groups * g.n_col_tiles * g.splits : 0;
 
     // The producer and MMA loops are run by all 32 lanes of their warp with warp-uniform operands; one elected lane
     // issues each asynchronous instruction.  (Issued from a single-lane branch, every tcgen05.mma cost the thread
@@ -476,11 +480,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_kernel_1cta(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, GemmArgs g)
 {
-    if (g.d_active && *g.d_active == 0) return;             // nothing left to decode
-    const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
-    const int m_groups = (M + BM - 1) / BM;
-    const int num_tiles = m_groups * g.n_col_tiles * g.splits;
-    if ((int)blockIdx.x >= num_tiles) return;
+    pdl_trigger();
+    if ((int)blockIdx.x >= ((g.M + BM - 1) / BM) * g.n_col_tiles * g.splits) return;     // beyond the tiles of even the largest row count
 
     const int BN = g.bn, STAGES = g.stages, HALF = BN >> 1;
     const int STAGE_BYTES = A_BYTES + BN * BK * 2;
@@ -512,6 +513,12 @@ gemm_kernel_1cta(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t n_bufs = (uint32_t)g.acc_bufs, buf_stride = 256;
     const bool swiglu = (g.mode == GEMM_SWIGLU);
     const int num_ctas = (int)gridDim.x;
+
+    pdl_wait();                                             // the kernel before this one has completed: global memory from here on
+    const bool live = !(g.d_active && *g.d_active == 0);    // nothing left to decode: the loops below find no tile
+    const int M = g.d_m ? min(*g.d_m, g.M) : g.M;
+    const int m_groups = (M + BM - 1) / BM;
+    const int num_tiles = live ? m_groups * g.n_col_tiles * g.splits : 0;
 
     if (warp == 0) {
         // ---------------- TMA producer
@@ -806,9 +813,8 @@ int32_t gemm_launch(const GemmPlan &p, const int32_t *d_m, const int32_t *d_acti
         const long long tiles1 = (long long)((g.M + BM - 1) / BM) * g.n_col_tiles * g.splits;
         const int sms = num_sms();
         const unsigned grid1 = (unsigned)(tiles1 < sms ? tiles1 : sms);
-        if (g.stats) gemm_kernel_1cta<true><<<grid1, kGemmThreads, smem1, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
-        else gemm_kernel_1cta<false><<<grid1, kGemmThreads, smem1, stream>>>(p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g);
-        SFS_LAUNCH_CHECK();
+        if (g.stats) SFS_CUDA(launch_pdl(gemm_kernel_1cta<true>, dim3(grid1), dim3(kGemmThreads), smem1, stream, p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g));
+        else SFS_CUDA(launch_pdl(gemm_kernel_1cta<false>, dim3(grid1), dim3(kGemmThreads), smem1, stream, p.tmA, p.tmB[0], p.tmB[1], p.tmB[2], g));
         return SFS_OK;
     }
     size_t smem = (size_t)g.stages * (g.mb * A_BYTES + (g.bn / 2) * BK * 2) + kBarBytes + kEpiStageBytes + 1024;
