@@ -396,6 +396,8 @@ __global__ void generate_init_kernel(const int32_t *prompt, int32_t *tokens, uin
 // host_active[0]: sequences still decoding; host_active[1]: denoising steps the device has finished in this generation
 __global__ void mirror_active_kernel(const int32_t *ctrl_active, int32_t *host_active, int32_t steps_done)
 {
+    pdl_wait();
+    pdl_trigger();
     host_active[1] = steps_done;
     __threadfence_system();
     host_active[0] = *ctrl_active;
@@ -799,8 +801,7 @@ int32_t sfs_generate_steps(sfs_session *s, int32_t n_steps, int32_t *d_trace, in
         a.ticket = s->ticket;
         a.trace = (d_trace && s->gen_steps < max_trace_steps) ? d_trace + (size_t)s->gen_steps * B * SFS_TRACE_INTS : nullptr;
         if ((rc = timed_launch(s, SFS_K_SELECT, st, [&] { return launch_select(a, st); })) != SFS_OK) return rc;
-        mirror_active_kernel<<<1, 1, 0, st>>>(s->ctrl + 2, s->host_active_dev, s->gen_steps + 1);
-        SFS_LAUNCH_CHECK();
+        SFS_CUDA(launch_pdl(mirror_active_kernel, dim3((unsigned)(1)), dim3((unsigned)(1)), (size_t)(0), st, s->ctrl + 2, s->host_active_dev, s->gen_steps + 1));
         s->launches++;
         s->gen_cur = nxt;
         s->gen_steps++;

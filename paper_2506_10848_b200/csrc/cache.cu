@@ -12,6 +12,8 @@ __global__ void __launch_bounds__(256)
 sim_partial_kernel(const __nv_bfloat16 *__restrict__ a, const __nv_bfloat16 *__restrict__ b, long long ld, int d, int t_first, int t_end, int T,
                    float *__restrict__ partial)
 {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int t0 = t_first + blockIdx.x * 64 + 2 * lane;             // t_first is even: 4-byte loads of two tokens stay aligned
     const int per = (d + kSimSlices - 1) / kSimSlices;
@@ -60,6 +62,8 @@ __device__ __forceinline__ uint32_t float_order_key(float f) {       // monotone
 // one CTA per sequence; dynamic shared memory: u64 keys[L], u8 chosen[L]
 __global__ void __launch_bounds__(1024) cache_select_kernel(CacheSelectArgs a)
 {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ unsigned long long s_key[];
     const int b = blockIdx.x, tid = threadIdx.x, L = a.L, P = a.P, S = a.S;
     int32_t *out = a.sel_rows + (long long)b * a.n_sel;
@@ -126,6 +130,8 @@ __global__ void __launch_bounds__(1024) cache_select_kernel(CacheSelectArgs a)
 
 __global__ void gather_rows_bf16_kernel(const uint4 *__restrict__ src, const int32_t *__restrict__ rows, int chunks, uint4 *__restrict__ dst)
 {
+    pdl_wait();
+    pdl_trigger();
     const int j = blockIdx.x;
     const uint4 *s = src + (long long)rows[j] * chunks;
     uint4 *o = dst + (long long)j * chunks;
@@ -135,6 +141,8 @@ __global__ void gather_rows_bf16_kernel(const uint4 *__restrict__ src, const int
 __global__ void scatter_rows_f32_kernel(const float4 *__restrict__ src, int n_slabs, long long slab_chunks, const int32_t *__restrict__ rows,
                                         int chunks, float4 *__restrict__ dst)
 {
+    pdl_wait();
+    pdl_trigger();
     const int j = blockIdx.x;
     const float4 *s = src + (long long)j * chunks;
     float4 *o = dst + (long long)rows[j] * chunks;
@@ -177,6 +185,8 @@ rope_scatter_kv_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int n_rows,
                        const int32_t *__restrict__ rows, __nv_bfloat16 *__restrict__ k_dst, const __nv_bfloat16 *__restrict__ vt_src,
                        long long ld_vt_src, __nv_bfloat16 *__restrict__ vt_dst, long long ld_vt_dst, int rope_blocks)
 {
+    pdl_wait();
+    pdl_trigger();
     const int d = n_heads * dh;
     if ((int)blockIdx.x >= rope_blocks) {
         const int f0 = ((int)blockIdx.x - rope_blocks) * 8;
@@ -232,6 +242,8 @@ fold_norm_rows_kernel(const float *__restrict__ slabs, int n_slabs, long long sl
                       const float *__restrict__ x, float *__restrict__ inc, const __nv_bfloat16 *__restrict__ gain,
                       __nv_bfloat16 *__restrict__ h, int d, float eps)
 {
+    pdl_wait();
+    pdl_trigger();
     const int j = blockIdx.x, chunks = d / 4;
     const long long src = rows[j];
     const float4 *sp = reinterpret_cast<const float4 *>(slabs + (long long)j * d);
@@ -279,10 +291,9 @@ int32_t launch_rope_scatter_kv(void *qk, long long ld, int n_rows, int S, int n_
     const long long total = (long long)n_rows * 2 * n_heads * (head_dim / 16);
     SFS_REQUIRE(total < (1LL << 31), SFS_ERR_INVALID_ARG, "rope: %lld items do not fit a 32-bit index", total);
     const int rope_blocks = (int)((total + 255) / 256), d = n_heads * head_dim;
-    rope_scatter_kv_kernel<<<rope_blocks + (d + 7) / 8, 256, 0, s>>>(reinterpret_cast<__nv_bfloat16 *>(qk), ld, n_rows, S, n_heads, head_dim, table, rows,
+    SFS_CUDA(launch_pdl(rope_scatter_kv_kernel, dim3((unsigned)(rope_blocks + (d + 7) / 8)), dim3((unsigned)(256)), (size_t)(0), s, reinterpret_cast<__nv_bfloat16 *>(qk), ld, n_rows, S, n_heads, head_dim, table, rows,
                                                                       reinterpret_cast<__nv_bfloat16 *>(k_dst), reinterpret_cast<const __nv_bfloat16 *>(vt_src),
-                                                                      ld_vt_src, reinterpret_cast<__nv_bfloat16 *>(vt_dst), ld_vt_dst, rope_blocks);
-    SFS_LAUNCH_CHECK();
+                                                                      ld_vt_src, reinterpret_cast<__nv_bfloat16 *>(vt_dst), ld_vt_dst, rope_blocks));
     return SFS_OK;
 }
 
@@ -293,9 +304,8 @@ int32_t launch_fold_norm_rows(const float *slabs, int n_slabs, long long slab_st
     SFS_REQUIRE((size_t)d * 4 <= 96 * 1024, SFS_ERR_UNSUPPORTED, "d_model %d too wide for the fused fold + norm", d);
     const size_t smem = (size_t)d * 4;
     if (smem > 48 * 1024) SFS_CUDA(cudaFuncSetAttribute(fold_norm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    fold_norm_rows_kernel<<<n_rows, 256, smem, s>>>(slabs, n_slabs < 1 ? 1 : n_slabs, slab_stride, rows, x, inc, reinterpret_cast<const __nv_bfloat16 *>(gain),
-                                                    reinterpret_cast<__nv_bfloat16 *>(h), d, eps);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(fold_norm_rows_kernel, dim3((unsigned)(n_rows)), dim3((unsigned)(256)), (size_t)(smem), s, slabs, n_slabs < 1 ? 1 : n_slabs, slab_stride, rows, x, inc, reinterpret_cast<const __nv_bfloat16 *>(gain),
+                                                    reinterpret_cast<__nv_bfloat16 *>(h), d, eps));
     return SFS_OK;
 }
 
@@ -305,25 +315,22 @@ int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld,
     if (t_count <= 0) return SFS_OK;
     SFS_REQUIRE((t_first % 2) == 0 && (ld % 2) == 0, SFS_ERR_INVALID_ARG, "similarity: first token and row stride must be even");
     dim3 grid((unsigned)((t_count + 63) / 64), kSimSlices, 1);
-    sim_partial_kernel<<<grid, 256, 0, s>>>(reinterpret_cast<const __nv_bfloat16 *>(vnew_t), reinterpret_cast<const __nv_bfloat16 *>(vold_t),
-                                            ld, d, t_first, t_first + t_count, T, partial);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(sim_partial_kernel, grid, dim3((unsigned)(256)), (size_t)(0), s, reinterpret_cast<const __nv_bfloat16 *>(vnew_t), reinterpret_cast<const __nv_bfloat16 *>(vold_t),
+                                            ld, d, t_first, t_first + t_count, T, partial));
     return SFS_OK;
 }
 
 int32_t launch_cache_select(const CacheSelectArgs &a, cudaStream_t s)
 {
     const int threads = a.L >= 512 ? 1024 : (a.L > 256 ? 512 : 256);         // the ranking is O(L^2 / threads)
-    cache_select_kernel<<<a.B, threads, (size_t)a.L * 9 + 16, s>>>(a);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(cache_select_kernel, dim3((unsigned)(a.B)), dim3((unsigned)(threads)), (size_t)((size_t)a.L * 9 + 16), s, a));
     return SFS_OK;
 }
 
 int32_t launch_gather_rows_bf16(const void *src, const int32_t *rows, int n_rows, int d, void *dst, cudaStream_t s)
 {
     if (n_rows <= 0) return SFS_OK;
-    gather_rows_bf16_kernel<<<n_rows, 128, 0, s>>>(reinterpret_cast<const uint4 *>(src), rows, d / 8, reinterpret_cast<uint4 *>(dst));
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(gather_rows_bf16_kernel, dim3((unsigned)(n_rows)), dim3((unsigned)(128)), (size_t)(0), s, reinterpret_cast<const uint4 *>(src), rows, d / 8, reinterpret_cast<uint4 *>(dst)));
     return SFS_OK;
 }
 
@@ -331,9 +338,8 @@ int32_t launch_scatter_rows_f32(const float *src, int n_slabs, long long slab_st
                                 cudaStream_t s)
 {
     if (n_rows <= 0) return SFS_OK;
-    scatter_rows_f32_kernel<<<dim3((unsigned)n_rows, 4, 1), 256, 0, s>>>(reinterpret_cast<const float4 *>(src), n_slabs < 1 ? 1 : n_slabs, slab_stride / 4, rows, d / 4,
-                                                   reinterpret_cast<float4 *>(dst));
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(scatter_rows_f32_kernel, dim3((unsigned)n_rows, 4, 1), dim3((unsigned)(256)), (size_t)(0), s, reinterpret_cast<const float4 *>(src), n_slabs < 1 ? 1 : n_slabs, slab_stride / 4, rows, d / 4,
+                                                   reinterpret_cast<float4 *>(dst)));
     return SFS_OK;
 }
 

@@ -10,6 +10,8 @@ namespace {
 __global__ void embed_kernel(const int32_t *__restrict__ tokens, const __nv_bfloat16 *__restrict__ emb,
                              float *__restrict__ x, int T, int d, int vocab)
 {
+    pdl_wait();
+    pdl_trigger();
     const int t = blockIdx.x;
     if (t >= T) return;
     int id = tokens[t];
@@ -158,8 +160,7 @@ __global__ void rope_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int T,
 
 int32_t launch_embed(const int32_t *tokens, const void *emb, float *x, int T, int d, int vocab, cudaStream_t s)
 {
-    embed_kernel<<<T, 128, 0, s>>>(tokens, reinterpret_cast<const __nv_bfloat16 *>(emb), x, T, d, vocab);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(embed_kernel, dim3((unsigned)(T)), dim3((unsigned)(128)), (size_t)(0), s, tokens, reinterpret_cast<const __nv_bfloat16 *>(emb), x, T, d, vocab));
     return SFS_OK;
 }
 

@@ -265,6 +265,8 @@ __device__ __forceinline__ uint32_t smem_addr(const void *p) { return (uint32_t)
 constexpr int kDecideThreads = 256;
 __global__ void __launch_bounds__(kDecideThreads) refine_decide_kernel(RefineArgs rf)
 {
+    pdl_wait();
+    pdl_trigger();
     const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, L = rf.L;
     const sfs_state &st = rf.state[b];
     if (st.done || st.status != SFS_OK) return;
@@ -503,6 +505,8 @@ __global__ void __launch_bounds__(128)
 combine_partials_kernel(const float4 *__restrict__ stats, int stats_ld, int n_parts, const int32_t *__restrict__ n_rows_ptr, int max_rows,
                         int vocab, BoundsOut out)
 {
+    pdl_wait();
+    pdl_trigger();
     const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     const int n_rows = n_rows_ptr ? min(*n_rows_ptr, max_rows) : max_rows;
     if (blockIdx.x == 0 && threadIdx.x == 0 && out.list_count) *out.list_count = 0;
@@ -692,6 +696,8 @@ rowstats_list_bf16(const uint4 *__restrict__ logits, long long ld_chunks, int nc
                    const int32_t *__restrict__ list, const int32_t *__restrict__ list_count, const float *__restrict__ pos_max,
                    unsigned long long *__restrict__ pos_sq, int n_positions)
 {
+    pdl_wait();
+    pdl_trigger();
     const int n_items = *list_count * kListParts;
     const int per = (nchunks + kListParts - 1) / kListParts;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -948,12 +954,10 @@ int32_t launch_row_stats_two_pass(const void *d_logits, int32_t vocab, int64_t l
                  reinterpret_cast<float4 *>(rf.slice_partials), rf.row_tickets};
     int32_t rc = launch_bounds(lp, ld / 8, vocab / 8, vocab, d_n_rows, max_rows, bo, stream);
     if (rc != SFS_OK) return rc;
-    refine_decide_kernel<<<rf.B, kDecideThreads, 0, stream>>>(rf);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(refine_decide_kernel, dim3((unsigned)(rf.B)), dim3((unsigned)(kDecideThreads)), (size_t)(0), stream, rf));
     const int items = max_rows * kListParts, cap = 2 * num_sms_rowstats();
-    rowstats_list_bf16<<<items < cap ? items : cap, kListThreads, 0, stream>>>(lp, ld / 8, vocab / 8, d_rows, rf.refine_list, rf.refine_count,
-                                                                              rf.pos_max, rf.pos_sq, rf.B * rf.S);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(rowstats_list_bf16, dim3((unsigned)(items < cap ? items : cap)), dim3((unsigned)(kListThreads)), (size_t)(0), stream, lp, ld / 8, vocab / 8, d_rows, rf.refine_list, rf.refine_count,
+                                                                              rf.pos_max, rf.pos_sq, rf.B * rf.S));
     return SFS_OK;
 }
 
@@ -964,15 +968,12 @@ int32_t launch_row_stats_from_partials(const void *stats, int32_t stats_ld, int3
     if (max_rows <= 0) return SFS_OK;
     BoundsOut bo{d_rows, nullptr, nullptr, nullptr, rf.pos_lo, rf.pos_hi, rf.pos_arg, rf.pos_row, rf.pos_max, rf.refine_count, rf.B * rf.S, d_err,
                  nullptr, nullptr};
-    combine_partials_kernel<<<(max_rows + 3) / 4, 128, 0, stream>>>(reinterpret_cast<const float4 *>(stats), stats_ld, n_parts, d_n_rows, max_rows, vocab, bo);
-    SFS_LAUNCH_CHECK();
-    refine_decide_kernel<<<rf.B, kDecideThreads, 0, stream>>>(rf);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(combine_partials_kernel, dim3((unsigned)((max_rows + 3) / 4)), dim3((unsigned)(128)), (size_t)(0), stream, reinterpret_cast<const float4 *>(stats), stats_ld, n_parts, d_n_rows, max_rows, vocab, bo));
+    SFS_CUDA(launch_pdl(refine_decide_kernel, dim3((unsigned)(rf.B)), dim3((unsigned)(kDecideThreads)), (size_t)(0), stream, rf));
     const uint4 *lp = reinterpret_cast<const uint4 *>(d_logits);
     const int items = max_rows * kListParts, cap = 2 * num_sms_rowstats();
-    rowstats_list_bf16<<<items < cap ? items : cap, kListThreads, 0, stream>>>(lp, ld / 8, vocab / 8, d_rows, rf.refine_list, rf.refine_count,
-                                                                              rf.pos_max, rf.pos_sq, rf.B * rf.S);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(rowstats_list_bf16, dim3((unsigned)(items < cap ? items : cap)), dim3((unsigned)(kListThreads)), (size_t)(0), stream, lp, ld / 8, vocab / 8, d_rows, rf.refine_list, rf.refine_count,
+                                                                              rf.pos_max, rf.pos_sq, rf.B * rf.S));
     return SFS_OK;
 }
 

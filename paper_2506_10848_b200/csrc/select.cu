@@ -75,6 +75,8 @@ __device__ __forceinline__ uint32_t philox_first_word(uint32_t c0, uint32_t c1, 
 // dynamic shared memory: keys u64[L] | flags u8[L] (selected) | flags u8[L] (above tau_high)
 __global__ void __launch_bounds__(kSelThreads) select_kernel(SelectArgs a)
 {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ unsigned long long s_keys[];
     const int L = a.L, S = a.S, P = a.P, b = blockIdx.x, tid = threadIdx.x;
     uint8_t *s_sel  = reinterpret_cast<uint8_t *>(s_keys + L);
@@ -302,8 +304,7 @@ int32_t launch_select(const SelectArgs &a, cudaStream_t stream)
     if (smem > 48 * 1024) {
         SFS_CUDA(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     }
-    select_kernel<<<a.B, kSelThreads, smem, stream>>>(a);
-    SFS_LAUNCH_CHECK();
+    SFS_CUDA(launch_pdl(select_kernel, dim3((unsigned)(a.B)), dim3((unsigned)(kSelThreads)), (size_t)(smem), stream, a));
     return SFS_OK;
 }
 
