@@ -147,3 +147,46 @@ def test_vanilla_generation_on_the_tiny_model_is_reproduced_by_the_oracle(strate
     finally:
         sfs.sfs_session_destroy(session)
         model.close()
+
+
+@pytest.mark.parametrize("strategy,N,bl", [(SM.LOW_CONFIDENCE, 0, 0), (SM.LOW_CONFIDENCE, 8, 12), (SM.RANDOM, 6, 0)])
+def test_vanilla_samplers_on_full_vocabulary_rows(strategy, N, bl):
+    """Long bf16 rows go through the two-pass row statistics, whose second pass must know what each strategy asks of a row
+    (low-confidence: the ranking, top-1 or top-k; random: nothing).  Confidences are planted close together so that the
+    ranking is decided by the canonical values."""
+    V, B, P, L = 126464, 2, 0, 24
+    S = P + L
+    po, pg = pair(strategy, N, bl, 77)
+    session = sfs.sfs_select_session_create(V, B, S)
+    try:
+        tokens = torch.full((B, S), V - 1, dtype=torch.int32, device=DEV)
+        mask = torch.ones((B, S), dtype=torch.uint8, device=DEV)
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+        sfs.sfs_state_init(state, B, L, pg)
+        sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+        sel_pos = torch.zeros((B, L), dtype=torch.int32, device=DEV); sel_tok = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+        ost = [SM.VanillaState.fresh(L, po) for _ in range(B)]
+        g = torch.Generator().manual_seed(5)
+        step = 0
+        while not all(s_.done for s_ in ost):
+            need = [(b, i) for b in range(B) for i in SM.vanilla_rows_needed(ost[b])]
+            conf = 0.3 + 2e-5 * torch.randint(0, 4, (max(len(need), 1),), generator=g).double()      # near-ties
+            logits = W.logits_for_confidences(conf, V, seed=9, step=step)
+            rows = torch.tensor([b * S + P + i for (b, i) in need] or [0], dtype=torch.int32, device=DEV)
+            n_dev = torch.tensor([len(need)], dtype=torch.int32, device=DEV)
+            sfs.sfs_select(session, logits.to(DEV), sfs.LOGITS_BF16, V, rows, n_dev, max(len(need), 1), tokens, mask, B, S, P, state, pg,
+                           sel_count, sel_pos, sel_tok)
+            torch.cuda.synchronize()
+            st = RS.row_stats(W.bf16_bits(logits))
+            for b in range(B):
+                if ost[b].done:
+                    continue
+                idx = {i: j for j, (bb, i) in enumerate(need) if bb == b}
+                rec = SM.vanilla_step(ost[b], {i: int(st["argmax"][j]) for i, j in idx.items()}, {i: int(st["sq"][j]) for i, j in idx.items()}, po, seq=b)
+                n = int(sel_count[b])
+                assert sel_pos[b, :n].tolist() == rec.positions and sel_tok[b, :n].tolist() == rec.tokens, (step, b)
+            step += 1
+        assert int(mask.sum()) == 0
+        sfs.sfs_check_device_status()
+    finally:
+        sfs.sfs_session_destroy(session)

@@ -243,14 +243,14 @@ def test_statistics_of_a_finished_sequence_do_not_survive_into_the_next_generati
         sfs.sfs_session_destroy(session)
 
 
-@pytest.mark.parametrize("case", ["near_ties", "threshold_edges", "all_confident"])
+@pytest.mark.parametrize("case", ["near_ties", "threshold_edges", "all_confident", "near_ties_k2"])
 def test_full_vocabulary_steps_where_the_cheap_pass_cannot_decide(case):
     """Long bf16 rows take the two-pass row statistics.  These inputs are built so that the enclosures of the cheap pass
     leave the step's questions open — top-1 candidates closer than the enclosure width, confidences within 1e-5 of a
     threshold, many rows with S_q = 2^28 exactly — and the decisions must still be the oracle's, slow and fast step."""
     V, L, P, B = 126464, 48, 0, 1
-    po, pg = params_pair()
-    if case == "near_ties":
+    po, pg = params_pair(k_slow=2, k_fast=3) if case == "near_ties_k2" else params_pair()     # k > 1: every candidate is recomputed
+    if case.startswith("near_ties"):
         conf = torch.full((L,), 0.05, dtype=torch.float64)
         conf[10] = 0.30000; conf[20] = 0.30001; conf[30] = 0.29999; conf[31] = 0.30000        # best four within 3e-5 relative
     elif case == "threshold_edges":
