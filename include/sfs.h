@@ -126,7 +126,9 @@ typedef struct {
 
 /* Section 3.1 (the mask predictor p_theta).  Checks shapes (head_dim 64 or 128, n_heads*head_dim == d_model,
  * d_model and d_ff multiples of 8, vocab a multiple of 8), copies the pointer tables and precomputes the
- * RoPE table.  Allocates device memory; synchronises. */
+ * RoPE table.  Allocates device memory; synchronises the device, so whatever wrote the weights has finished.
+ * The weight arrays stay the caller's: they must outlive the model and must not be written while a call that
+ * uses the model is in flight. */
 int32_t sfs_model_create(const sfs_config *cfg, const sfs_weights *weights, sfs_model **out);
 int32_t sfs_model_destroy(sfs_model *model);
 

@@ -468,6 +468,8 @@ int32_t sfs_model_create(const sfs_config *cfg, const sfs_weights *w, sfs_model 
         m->w_down.push_back(ps[8]);
     }
     if (!ok) { delete m; set_error("model_create: every weight pointer must be non-NULL and 16-byte aligned"); return SFS_ERR_INVALID_ARG; }
+    // whatever wrote the weights (on any stream) has finished before a forward pass on another stream reads them
+    if (cudaDeviceSynchronize() != cudaSuccess) { delete m; set_error("model_create: device synchronisation failed"); return SFS_ERR_CUDA; }
     *out = m;
     return SFS_OK;
 }
