@@ -26,8 +26,10 @@ def max_abs_bar(logit_scale):
     return MAX_ABS * max(1.0, logit_scale / 4.0)
 
 
-@pytest.mark.parametrize("B,S,H,dh", [(1, 96, 4, 64), (2, 136, 2, 128), (1, 512, 2, 128), (3, 264, 1, 64), (2, 768, 2, 128), (1, 1536, 1, 128)])
+@pytest.mark.parametrize("B,S,H,dh", [(1, 96, 4, 64), (2, 136, 2, 128), (1, 512, 2, 128), (3, 264, 1, 64), (2, 768, 2, 128), (1, 1536, 1, 128),
+                                      (1, 1024, 2, 64), (1, 648, 1, 64), (1, 1160, 3, 128)])
 def test_attention_matches_oracle(B, S, H, dh):
+    # up to 12 key tiles per query tile, ragged last tiles (96, 136, 264, 648, 1160), both head dimensions
     g = torch.Generator().manual_seed(S + dh)
     d = H * dh
     q = torch.randn((B * S, d), generator=g).to(torch.bfloat16)
