@@ -527,6 +527,8 @@ def main():
     ap.add_argument("--no-extras", dest="extras", action="store_false", help="skip the epilogue / cached / batch-8 workloads")
     ap.add_argument("--no-cpu-baseline", dest="cpu", action="store_false")
     ap.add_argument("--epilogue-only", action="store_true", help="run only the sampling-epilogue microbenchmark (small case for ncu captures)")
+    ap.add_argument("--cached-only", action="store_true",
+                    help="run only a few feature-cache steps (prompt 1024 + 512 masked, K_p 100, K_r 5; with --layers: a small case for ncu launch lists)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", 0))
@@ -552,6 +554,31 @@ def main():
             from paper_2506_10848_b200 import workloads as W
             torch.cuda.set_device(0)
             print(json.dumps({"profiling_case": "sampling epilogue only", **run_epilogue(torch, sfs, W, W.LLADA_8B, "cuda:0", measured_peaks())}))
+        return
+    if args.cached_only:
+        # a profiling case, not a bench line: a full refresh, four partial steps, a response refresh and one more partial step
+        if rank == 0:
+            from paper_2506_10848_b200 import binding as sfs
+            from paper_2506_10848_b200 import workloads as W
+            torch.cuda.set_device(0)
+            shape = W.with_layers(W.LLADA_8B, args.layers) if args.layers else W.LLADA_8B
+            model = sfs.Model(shape, W.model_weights(shape, seed=2, device="cuda:0"))
+            session = sfs.sfs_session_create(model, 1, 1536)
+            prompt = W.prompt_ids(1, 1024, shape.vocab - 2, seed=3).to("cuda:0")
+            sfs.sfs_cache_enable(session, 100, 5, 0.25)
+            sfs.sfs_generate_begin(session, prompt, 1, 1024, 512, sfs.Params.default())
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            sfs.sfs_generate_steps(session, 1, None, 0)
+            e0.record()
+            sfs.sfs_generate_steps(session, 4, None, 0)
+            e1.record()
+            sfs.sfs_generate_steps(session, 2, None, 0)
+            torch.cuda.synchronize()
+            sfs.sfs_check_device_status()
+            print(json.dumps({"profiling_case": "feature-cache steps only", "layers": shape.n_layers,
+                              "cached_partial_step_ms": e0.elapsed_time(e1) / 4}))
+            sfs.sfs_session_destroy(session)
+            model.close()
         return
     res = run_ours(args, rank, world)
 

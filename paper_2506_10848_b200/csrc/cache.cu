@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(1024) cache_select_kernel(CacheSelectArgs a)
 {
     pdl_wait();
     pdl_trigger();
-    extern __shared__ unsigned long long s_key[];
+    extern __shared__ __align__(16) unsigned long long s_key[];
     const int b = blockIdx.x, tid = threadIdx.x, L = a.L, P = a.P, S = a.S;
     int32_t *out = a.sel_rows + (long long)b * a.n_sel;
     int base = 0;
@@ -95,30 +95,52 @@ __global__ void __launch_bounds__(1024) cache_select_kernel(CacheSelectArgs a)
             if (a.sims_dump) a.sims_dump[(long long)b * L + i] = sim;
             s_key[i] = (i >= lo && i < hi) ? (((unsigned long long)float_order_key(sim) << 32) | (unsigned)i) : ~0ull;
         }
+        const int Lp = (L + 1) & ~1;                               // keys are scanned two at a time: an odd L gets a sentinel
+        if (tid == 0 && Lp != L) s_key[L] = ~0ull;
         __syncthreads();
         const int n_cand = hi - lo;
         const int k = min(a.n_adapt, n_cand);
-        __shared__ int s_last;
+        __shared__ int s_last, s_wcnt[32];
         if (tid == 0) s_last = -1;
-        __syncthreads();
-        // rank by counting: candidate i is chosen when fewer than k candidate keys are smaller
-        uint8_t *s_sel = reinterpret_cast<uint8_t *>(s_key + L);
-        for (int i = tid; i < L; i += blockDim.x) {
-            const unsigned long long ki = s_key[i];
+        // rank by counting: candidate i is chosen when fewer than k candidate keys are smaller.  `parts` adjacent lanes share
+        // a candidate, each counting over its own range of the keys (16-byte loads, two keys each).
+        uint8_t *s_sel = reinterpret_cast<uint8_t *>(s_key + Lp);
+        int parts = 1;
+        while (parts < 32 && (long long)L * parts * 2 <= (long long)blockDim.x) parts *= 2;
+        const int span = ((Lp / 2 + parts - 1) / parts) * 2;      // keys per part (even)
+        const ulonglong2 *k2 = reinterpret_cast<const ulonglong2 *>(s_key);
+        const int items = ((L * parts + 31) / 32) * 32;           // whole warps take part in the shuffles
+        for (int it = tid; it < items; it += blockDim.x) {
+            const int i = it / parts, part = it - i * parts;
+            const unsigned long long ki = i < L ? s_key[i] : ~0ull;
             int rank = 0;
-            if (ki != ~0ull) for (int j = 0; j < L; ++j) rank += (s_key[j] < ki) ? 1 : 0;
-            s_sel[i] = (ki != ~0ull && rank < k) ? 1 : 0;
+            if (ki != ~0ull) {
+                const int j0 = part * span, j1 = min(Lp, j0 + span);
+                for (int j = j0; j < j1; j += 2) { const ulonglong2 kk = k2[j >> 1]; rank += (kk.x < ki ? 1 : 0) + (kk.y < ki ? 1 : 0); }
+            }
+            for (int o = 1; o < parts; o <<= 1) rank += __shfl_xor_sync(0xffffffffu, rank, o);
+            if (part == 0 && i < L) s_sel[i] = (ki != ~0ull && rank < k) ? 1 : 0;
         }
         __syncthreads();
-        // its slot in the ascending list is the number of chosen positions before it
-        for (int i = tid; i < L; i += blockDim.x) {
-            if (!s_sel[i]) continue;
-            int slot = 0;
-            for (int j = 0; j < i; ++j) slot += s_sel[j];
-            out[base + slot] = b * S + P + i;
-            if (slot == k - 1) s_last = b * S + P + i;
+        // its slot in the ascending list is the number of chosen positions before it (ballots and per-warp counts)
+        const int lane = tid & 31, warp = tid >> 5, n_warps = (int)blockDim.x >> 5;
+        int run = 0;
+        for (int i0 = 0; i0 < L; i0 += blockDim.x) {
+            const int i = i0 + tid;
+            const bool chosen = i < L && s_sel[i] != 0;
+            const unsigned bal = __ballot_sync(0xffffffffu, chosen);
+            if (lane == 0) s_wcnt[warp] = __popc(bal);
+            __syncthreads();
+            int before = run, total = 0;
+            for (int w = 0; w < n_warps; ++w) { const int cnt = s_wcnt[w]; total += cnt; if (w < warp) before += cnt; }
+            if (chosen) {
+                const int slot = before + __popc(bal & ((1u << lane) - 1u));
+                out[base + slot] = b * S + P + i;
+                if (slot == k - 1) s_last = b * S + P + i;
+            }
+            run += total;
+            __syncthreads();
         }
-        __syncthreads();
         const int pad = (k > 0) ? s_last : b * S + P;                  // nothing to choose from: recompute the first response row
         for (int j = k + tid; j < a.n_adapt; j += blockDim.x) out[base + j] = pad;
     }
@@ -237,7 +259,7 @@ rope_scatter_kv_kernel(__nv_bfloat16 *__restrict__ qk, long long ld, int n_rows,
 // One launch for what follows the output projection of the recomputed rows: the split-K slabs of compact row j are added in
 // slab order into the attention increment of its token (inc[rows[j]] = sum of slabs), and the MLP branch's input
 // h[j] = bf16(RMSNorm(x[rows[j]] + inc[rows[j]]) * gain) is written to the compact buffer.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(1024)
 fold_norm_rows_kernel(const float *__restrict__ slabs, int n_slabs, long long slab_stride, const int32_t *__restrict__ rows,
                       const float *__restrict__ x, float *__restrict__ inc, const __nv_bfloat16 *__restrict__ gain,
                       __nv_bfloat16 *__restrict__ h, int d, float eps)
@@ -249,7 +271,7 @@ fold_norm_rows_kernel(const float *__restrict__ slabs, int n_slabs, long long sl
     const float4 *sp = reinterpret_cast<const float4 *>(slabs + (long long)j * d);
     const float4 *xr = reinterpret_cast<const float4 *>(x + src * d);
     float4 *ir = reinterpret_cast<float4 *>(inc + src * d);
-    __shared__ float s_part[8];
+    __shared__ float s_part[32];
     extern __shared__ float4 s_y[];                            // the row, kept between the two passes
     float ss = 0.f;
     for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
@@ -268,8 +290,7 @@ fold_norm_rows_kernel(const float *__restrict__ slabs, int n_slabs, long long sl
     if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) tot += s_part[w];
+    for (int w = 0; w < ((int)blockDim.x >> 5); ++w) tot += s_part[w];
     const float inv = rsqrtf(tot / (float)d + eps);
     const uint2 *gp = reinterpret_cast<const uint2 *>(gain);
     uint2 *hp = reinterpret_cast<uint2 *>(h + (long long)j * d);
@@ -304,7 +325,7 @@ int32_t launch_fold_norm_rows(const float *slabs, int n_slabs, long long slab_st
     SFS_REQUIRE((size_t)d * 4 <= 96 * 1024, SFS_ERR_UNSUPPORTED, "d_model %d too wide for the fused fold + norm", d);
     const size_t smem = (size_t)d * 4;
     if (smem > 48 * 1024) SFS_CUDA(cudaFuncSetAttribute(fold_norm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    SFS_CUDA(launch_pdl(fold_norm_rows_kernel, dim3((unsigned)(n_rows)), dim3((unsigned)(256)), (size_t)(smem), s, slabs, n_slabs < 1 ? 1 : n_slabs, slab_stride, rows, x, inc, reinterpret_cast<const __nv_bfloat16 *>(gain),
+    SFS_CUDA(launch_pdl(fold_norm_rows_kernel, dim3((unsigned)(n_rows)), dim3((unsigned)(d >= 4096 ? 1024 : (d >= 2048 ? 512 : 256))), (size_t)(smem), s, slabs, n_slabs < 1 ? 1 : n_slabs, slab_stride, rows, x, inc, reinterpret_cast<const __nv_bfloat16 *>(gain),
                                                     reinterpret_cast<__nv_bfloat16 *>(h), d, eps));
     return SFS_OK;
 }
@@ -322,8 +343,8 @@ int32_t launch_sim_partial(const void *vnew_t, const void *vold_t, long long ld,
 
 int32_t launch_cache_select(const CacheSelectArgs &a, cudaStream_t s)
 {
-    const int threads = a.L >= 512 ? 1024 : (a.L > 256 ? 512 : 256);         // the ranking is O(L^2 / threads)
-    SFS_CUDA(launch_pdl(cache_select_kernel, dim3((unsigned)(a.B)), dim3((unsigned)(threads)), (size_t)((size_t)a.L * 9 + 16), s, a));
+    // 1024 threads: the ranking is O(L^2 / threads); shared memory: the keys (an even number of them), then one byte per position
+    SFS_CUDA(launch_pdl(cache_select_kernel, dim3((unsigned)(a.B)), dim3((unsigned)(1024)), (size_t)((size_t)(a.L + 1) * 9 + 16), s, a));
     return SFS_OK;
 }
 
