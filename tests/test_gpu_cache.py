@@ -37,7 +37,8 @@ def check_logits(got, ref, scale):
 # (1, 512, 128, ..): a long sequence (five key tiles) and few recomputed rows: a compact query tile against many cached key
 # tiles; (1, 9, 55, ..): an odd prompt length (the response starts at an odd token index)
 @pytest.mark.parametrize("B,P,L,kp,kr,rho", [(1, 32, 64, 100, 3, 0.25), (2, 24, 40, 4, 2, 0.3), (1, 8, 56, 5, 100, 0.1),
-                                             (1, 512, 128, 100, 4, 0.25), (1, 9, 55, 100, 3, 0.2)])
+                                             (1, 512, 128, 100, 4, 0.25), (1, 9, 55, 100, 3, 0.2),
+                                             (1, 8, 1112, 100, 3, 0.1)])      # more response positions than the choice kernel has threads
 def test_cached_steps_match_oracle_under_the_same_schedule(B, P, L, kp, kr, rho):
     shape, model, cfg, w64 = tiny_setup(seed=3)
     S = P + L
