@@ -427,6 +427,43 @@ def run_extras(torch, sfs, W, model, shape, dev, peaks, weights=None):
         sfs.sfs_session_destroy(session)
         m2.close()
         torch.cuda.empty_cache()
+
+        # ---- context for the GEMM roofline: the library's GEMM (torch.matmul, i.e. cuBLAS) on the same weights at the same row
+        # counts, one call per weight matrix, 32 layers back to back (every pass streams the 13 GB of layer weights, as a step does).
+        # Not part of the path and not a target: it says what the measured-peak denominator turns into at these shapes.
+        d, ff, nl = shape.d_model, shape.d_ff, shape.n_layers
+        lib = {}
+        for T in (512, 6144):
+            x = torch.randn((T, d), device=dev, dtype=torch.float32).to(torch.bfloat16)
+            hid = torch.randn((T, ff), device=dev, dtype=torch.float32).to(torch.bfloat16)
+            o_d = torch.empty((T, d), device=dev, dtype=torch.bfloat16)
+            o_ff = torch.empty((T, ff), device=dev, dtype=torch.bfloat16)
+
+            def one_pass():
+                for lw in weights["layers"]:
+                    for name in ("wq", "wk", "wv", "wo"):
+                        torch.matmul(x, lw[name].t(), out=o_d)
+                    torch.matmul(x, lw["w_gate"].t(), out=o_ff)
+                    torch.matmul(x, lw["w_up"].t(), out=o_ff)
+                    torch.matmul(hid, lw["w_down"].t(), out=o_d)
+
+            n_pass = 160 if T == 512 else 16                   # about a second each: under the power cap like the timed step
+            one_pass(); one_pass()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(n_pass):
+                one_pass()
+            e1.record()
+            torch.cuda.synchronize()
+            ms_pass = e0.elapsed_time(e1) / n_pass
+            fl = 2.0 * T * (4 * d * d + 3 * d * ff) * nl
+            lib[f"rows_{T}"] = {"ms_per_pass": ms_pass, "tflops": fl / (ms_pass * 1e-3) / 1e12, "gemm_calls_per_pass": 7 * nl}
+            del x, hid, o_d, o_ff
+        lib["note"] = ("torch.matmul (cuBLAS) bf16 on the layer weights, 7 calls per layer, no fusion, outputs discarded, about one second "
+                       "per row count; context for roofline.achieved, whose kernels also do the SwiGLU, residual and transposed-V epilogues")
+        out["library_gemm_context"] = lib
+        torch.cuda.empty_cache()
     return out
 
 
