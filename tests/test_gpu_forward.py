@@ -93,15 +93,21 @@ def test_forward_logits_tiny_within_tolerance():
         model.close()
 
 
-@pytest.mark.parametrize("logit_scale,B", [(8.0, 1), (60.0, 3)])
-def test_generate_tiny_teacher_forced(logit_scale, B):
+@pytest.mark.parametrize("logit_scale,B,P,L,pkw", [
+    (8.0, 1, 32, 64, {}), (60.0, 3, 32, 64, {}),
+    (60.0, 1, 0, 8, {}),                         # no prompt at all
+    (60.0, 2, 7, 1, {}),                         # a single position to decode
+    (60.0, 1, 5, 19, {"max_steps": 3}),          # the step budget runs out long before the positions do
+    (8.0, 2, 3, 13, {"max_steps": 4, "k_slow": 2, "k_fast": 3}),
+])
+def test_generate_tiny_teacher_forced(logit_scale, B, P, L, pkw):
     """Whole loop on the device; then the oracle's selection is fed the GPU's own logits step by step and
     must reproduce the GPU's trace and tokens exactly.  logit_scale 60 makes confidences cross both
-    thresholds, so parallel unmasking and span logic are exercised with a real model in the loop."""
+    thresholds, so parallel unmasking and span logic are exercised with a real model in the loop.  The
+    degenerate shapes: empty prompt, one position, a budget of steps far below the number of positions."""
     shape, model, cfg, w64 = tiny_setup(logit_scale=logit_scale)
-    P, L = 32, 64
     S = P + L
-    po, pg = params_pair()
+    po, pg = params_pair(**pkw)
     prompt = W.prompt_ids(B, P, 4094, seed=0)
     session = sfs.sfs_session_create(model, B, S)
     try:
@@ -151,7 +157,7 @@ def test_generate_tiny_teacher_forced(logit_scale, B):
             assert tk[b, P:].tolist() == oy[b]
             assert steps_gpu[b] == ost[b].steps_done
         print("steps per sequence:", steps_gpu)
-        if logit_scale > 30:
+        if logit_scale > 30 and L >= 32 and not pkw:
             assert min(steps_gpu) < L                      # thresholds fired: fewer steps than tokens
 
         # first-step logits against the oracle's own forward (the response is fully masked at step 0)
