@@ -10,6 +10,7 @@ from oracle.scheduler import SlowFastParams
 from paper_2506_10848_b200 import binding as sfs
 from paper_2506_10848_b200 import workloads as W
 
+from bf16_reference import forward_bf16_points
 from helpers import params_pair, state_to_dict
 
 pytestmark = pytest.mark.gpu
@@ -90,6 +91,52 @@ def test_forward_logits_tiny_within_tolerance():
         assert float(lgb[n - 3:].abs().max()) == 0.0
     finally:
         sfs.sfs_session_destroy(session)
+        model.close()
+
+
+@pytest.mark.parametrize("dims", [dict(d_model=384, n_heads=3, head_dim=128, d_ff=1000, vocab=5000),
+                                  dict(d_model=640, n_heads=10, head_dim=64, d_ff=1736, vocab=8200)])
+def test_forward_logits_at_widths_that_fill_no_tile(dims):
+    """Widths that are multiples of 8 and of nothing larger where the library allows it (d_ff, vocab), three or ten heads, a
+    sequence of 72 or 200 tokens: ragged tiles in every projection (rows, columns and the K of the down projection), ragged
+    key tiles, and a vocabulary that ends inside a column tile."""
+    shape = W.Shape(n_layers=2, mask_id=dims["vocab"] - 1, rms_eps=1e-5, rope_theta=10000.0, logit_scale=8.0, **dims)
+    w = W.model_weights(shape, seed=5)
+    wd = {k: (v.to(DEV) if k != "layers" else [{kk: vv.to(DEV) for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
+    model = sfs.Model(shape, wd)
+    cfg = F.ModelConfig(**shape.asdict())
+    w64 = W.weights_to_numpy(w, np.float64)
+    try:
+        for (B, P, L) in ((2, 31, 41), (1, 9, 191)):
+            S = P + L
+            tok = torch.cat([W.prompt_ids(B, P, shape.vocab - 2, seed=1), torch.full((B, L), shape.mask_id, dtype=torch.int32)], dim=1)
+            session = sfs.sfs_session_create(model, B, S)
+            rows = [(b, t) for b in range(B) for t in range(0, S, 5)]
+            d_rows = torch.tensor([b * S + t for (b, t) in rows], dtype=torch.int32, device=DEV)
+            lg = torch.zeros((len(rows), shape.vocab), dtype=torch.float32, device=DEV)
+            sfs.sfs_forward(session, tok.to(DEV), B, S, d_rows, None, len(rows), lg, sfs.LOGITS_F32)
+            sfs.sfs_check_device_status()
+            ref = F.forward(cfg, w64, tok.numpy(), rows=rows, dtype=np.float64)
+            got = lg.cpu().double().numpy()
+            rel_l2 = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+            # these logits are larger than the tiny model's (rms 4), so the absolute bar is the one of the rounding-only model
+            # of a bf16 pipeline (fp32 arithmetic, bf16 at the stored operands) against the same oracle, plus 30 %
+            emu = np.concatenate([forward_bf16_points(cfg, w, tok[b].numpy(), [t for (bb, t) in rows if bb == b]) for b in range(B)])
+            rel_model, abs_model = np.linalg.norm(emu - ref) / np.linalg.norm(ref), np.abs(emu - ref).max()
+            assert rel_l2 <= REL_L2 and rel_l2 <= 1.10 * rel_model, (B, S, rel_l2, rel_model)
+            assert np.abs(got - ref).max() <= 1.3 * abs_model, (B, S, np.abs(got - ref).max(), abs_model)
+            # and the whole loop runs to the end on this shape: every position decoded once, prompt untouched
+            out = torch.zeros((B, S), dtype=torch.int32, device=DEV)
+            state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+            sfs.sfs_generate(session, tok[:, :P].contiguous().to(DEV), B, P, L, sfs.Params.default(), out, state)
+            sfs.sfs_check_device_status()
+            o = out.cpu()
+            assert torch.equal(o[:, :P], tok[:, :P]) and int((o[:, P:] == shape.mask_id).sum()) == 0
+            for b in range(B):
+                st = state_to_dict(state[b])
+                assert st["done"] == 1 and st["n_masked"] == 0 and st["status"] == 0
+            sfs.sfs_session_destroy(session)
+    finally:
         model.close()
 
 
