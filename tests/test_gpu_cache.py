@@ -239,3 +239,45 @@ def test_cached_generation_is_reproduced_by_the_oracle_step_by_step(B, kp, kr, r
         assert n_unmasked == [L] * B and steps < L                 # finished, with parallel unmasking on the way
     finally:
         model.close()
+
+
+def test_cached_steps_at_widths_that_fill_no_tile():
+    """Three heads of 128, d_ff 1000, vocabulary 5000, 23 + 49 tokens: the few-row projections, gathers and scatters of the
+    partial steps with ragged tiles everywhere.  The tokens do not change, so the cached features stay exact and every step's
+    response logits must equal the uncached forward pass (oracle and GPU)."""
+    shape = W.Shape(n_layers=2, d_model=384, n_heads=3, head_dim=128, d_ff=1000, vocab=5000, mask_id=4999, rms_eps=1e-5,
+                    rope_theta=10000.0, logit_scale=8.0)
+    w = W.model_weights(shape, seed=6)
+    wd = {k: (v.to(DEV) if k != "layers" else [{kk: vv.to(DEV) for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
+    model = sfs.Model(shape, wd)
+    cfg = F.ModelConfig(**shape.asdict())
+    w64 = W.weights_to_numpy(w, np.float64)
+    B, P, L = 1, 23, 49
+    S = P + L
+    tok = torch.cat([W.prompt_ids(B, P, shape.vocab - 2, seed=2), torch.full((B, L), shape.mask_id, dtype=torch.int32)], dim=1)
+    d_tok = tok.to(DEV)
+    session = sfs.sfs_session_create(model, B, S)
+    try:
+        ref = F.forward(cfg, w64, tok.numpy(), rows=[(0, t) for t in range(S)], dtype=np.float64)
+        plain = torch.zeros((B * S, shape.vocab), dtype=torch.float32, device=DEV)
+        sfs.sfs_forward(session, d_tok, B, S, None, None, B * S, plain, sfs.LOGITS_F32)
+        plain = plain.cpu().double().numpy()
+        scale = np.abs(ref).max()
+        sfs.sfs_cache_enable(session, 100, 3, 0.3)
+        logits = torch.zeros((B * S, shape.vocab), dtype=torch.float32, device=DEV)
+        for step in range(6):
+            fast = step in (2, 4)
+            st = state_tensor(B, 1, 10, 31) if fast else state_tensor(B)
+            n_sel = sfs.sfs_forward_cached(session, d_tok, B, S, P, st, None, None, B * S, logits, sfs.LOGITS_F32)
+            sfs.sfs_check_device_status()
+            assert n_sel == (S if step == 0 else (L if step % 3 == 0 else C.adaptive_count(0.3, L)))
+            got = logits.cpu().double().numpy()
+            lo = 0 if step == 0 else P                       # prompt rows are defined on the step that refreshes the prompt
+            rel = np.linalg.norm(got[lo:] - ref[lo:]) / np.linalg.norm(ref[lo:])
+            rel_plain = np.linalg.norm(got[lo:] - plain[lo:]) / np.linalg.norm(plain[lo:])
+            assert rel <= REL_L2, (step, rel)
+            # the same features through other tile shapes and sum orders: far inside the rounding noise of either path
+            assert rel_plain <= 3e-3 and np.abs(got[lo:] - plain[lo:]).max() <= 2e-2 * scale, (step, rel_plain)
+    finally:
+        sfs.sfs_session_destroy(session)
+        model.close()
