@@ -47,10 +47,15 @@ def philox4x32_10(counter: Sequence[int], key: Sequence[int]) -> Tuple[int, int,
     return c0, c1, c2, c3
 
 
+def draw_accepts(u: int, k: int) -> bool:
+    """Whether the 32-bit draw u unmasks at countdown k: u / 2^32 < 1 / k, i.e. exactly ceil(2^32 / k) of the 2^32 values do."""
+    return u * k < (1 << 32)
+
+
 def random_unmask(seed: int, seq: int, step_index: int, position: int, k: int) -> bool:
     """One Bernoulli(1/k) draw of random remasking: position `position` of sequence `seq` at step index N - k."""
     u = philox4x32_10((position, step_index, seq, 0), (seed & M32, (seed >> 32) & M32))[0]
-    return u * k < (1 << 32)
+    return draw_accepts(u, k)
 
 
 # ---- the strategies, whole loops -------------------------------------------------------------------------------

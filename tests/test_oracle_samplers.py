@@ -121,6 +121,17 @@ def test_random_draw_is_the_integer_threshold_on_the_first_output_word():
     assert all(SM.random_unmask(5, 0, s, i, 1) for s in range(3) for i in range(40))      # k = 1: probability 1
 
 
+def test_a_draw_is_accepted_by_exactly_ceil_2_32_over_k_values():
+    """Random remasking unmasks with probability 1 - s/t = 1/k at countdown k (Section 3.1 with the linear schedule): the
+    accepted draws are u = 0 .. ceil(2^32 / k) - 1, also where k divides 2^32 and the boundary value is an integer."""
+    for k in (1, 2, 3, 4, 7, 256, 1000, 65536):
+        n_accept = -(-(1 << 32) // k)
+        assert SM.draw_accepts(n_accept - 1, k)
+        assert n_accept == (1 << 32) or not SM.draw_accepts(n_accept, k)
+        assert SM.draw_accepts(0, k)
+    assert not SM.draw_accepts((1 << 31), 2) and SM.draw_accepts((1 << 31) - 1, 2)
+
+
 @pytest.mark.parametrize("strategy", [SM.LOW_CONFIDENCE, SM.RANDOM])
 def test_semi_autoregressive_blocks_run_left_to_right(strategy):
     L, N, bl = 22, 12, 8                                    # blocks [0,8) [8,16) [16,22); 4 steps each
