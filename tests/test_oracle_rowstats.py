@@ -79,6 +79,28 @@ def test_power_of_two_gaps_closed_form():
         assert int(st["argmax"][0]) == V // 3
 
 
+def test_small_terms_truncate_to_the_integer_the_mathematics_fixes():
+    """A row {0, d}: S_q = 2^28 + trunc(2^28 e^d up to the recipe's 1e-5 relative error).  Where 2^28 e^d sits well inside an
+    integer interval the truncation is fixed by the mathematics alone: the terms just above 1 (the last shift that keeps a
+    bit), the first ones that vanish, and a ladder of small integers in between."""
+    ln2 = math.log(2.0)
+    checked = 0
+    for j in range(-3, 14):                                           # 2^28 e^d = 2^j * e^f
+        for f in (0.05, 0.2, 0.3):
+            d = np.float32(-(28 - j) * ln2 + f)
+            val = (1 << Q) * math.exp(float(d))                       # on the fp32 value actually handed over
+            if abs(val - round(val)) < 1e-4 * val + 0.02:             # too close to an integer to be fixed within 1e-5
+                continue
+            st = RS.row_stats(np.array([[0.0, d]], np.float32))
+            assert int(st["sq"][0]) == (1 << Q) + int(math.floor(val)), (j, f, val)
+            checked += 1
+    assert checked >= 40
+    # the three regimes by name: one unit left, nothing left, and exactly nothing far below
+    assert int(RS.row_stats(np.array([[0.0, -28 * ln2 + 0.2]], np.float32))["sq"][0]) == (1 << Q) + 1
+    assert int(RS.row_stats(np.array([[0.0, -29 * ln2 + 0.2]], np.float32))["sq"][0]) == (1 << Q)
+    assert int(RS.row_stats(np.array([[5.0, 5.0 - 28 * ln2 - 0.2]], np.float32))["sq"][0]) == (1 << Q)
+
+
 def test_canonical_sum_is_permutation_invariant_and_translation_stable():
     rng = np.random.default_rng(3)
     row = rng.normal(0, 4, 5000).astype(np.float32)
