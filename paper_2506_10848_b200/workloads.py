@@ -58,10 +58,19 @@ def normal_bf16(shape, std: float, seed: int, name: str, device: str = "cpu") ->
     return out
 
 
-def model_weights(shape: Shape, seed: int, device: str = "cpu", std: float = 0.02) -> Dict:
-    """Random-init weights: matrices N(0, std^2) as bf16, RMSNorm gains 1."""
+def model_weights(shape: Shape, seed: int, device: str = "cpu", std: float = 0.02, gain_std: float = 0.0) -> Dict:
+    """Random-init weights: matrices N(0, std^2) as bf16; RMSNorm gains 1, or 1 + N(0, gain_std^2) (each norm its own draw:
+    what the parity tests use, so that a gain that is dropped or taken from the wrong norm shows)."""
     d, ff, V = shape.d_model, shape.d_ff, shape.vocab
-    ones = lambda: torch.ones(d, dtype=torch.bfloat16, device=device)
+    count = [0]
+
+    def ones():
+        count[0] += 1
+        g = torch.ones(d, dtype=torch.float32, device=device)
+        if gain_std > 0.0:
+            g = g + normal_bf16((d,), gain_std, seed, f"gain{count[0]}", device).to(torch.float32)
+        return g.to(torch.bfloat16)
+
     w = {
         "tok_emb": normal_bf16((V, d), std, seed, "tok_emb", device),
         "final_norm": ones(),

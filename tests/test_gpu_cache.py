@@ -247,7 +247,7 @@ def test_cached_steps_at_widths_that_fill_no_tile():
     response logits must equal the uncached forward pass (oracle and GPU)."""
     shape = W.Shape(n_layers=2, d_model=384, n_heads=3, head_dim=128, d_ff=1000, vocab=5000, mask_id=4999, rms_eps=1e-5,
                     rope_theta=10000.0, logit_scale=8.0)
-    w = W.model_weights(shape, seed=6)
+    w = W.model_weights(shape, seed=6, gain_std=0.2)
     wd = {k: (v.to(DEV) if k != "layers" else [{kk: vv.to(DEV) for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
     model = sfs.Model(shape, wd)
     cfg = F.ModelConfig(**shape.asdict())

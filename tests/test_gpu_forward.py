@@ -55,7 +55,7 @@ def tiny_setup(seed=0, logit_scale=None):
     if logit_scale is not None:
         dct = shape.asdict(); dct["logit_scale"] = logit_scale
         shape = W.Shape(**dct)
-    w = W.model_weights(shape, seed=seed)
+    w = W.model_weights(shape, seed=seed, gain_std=0.2)       # every norm its own gains
     wd = {k: (v.to(DEV) if k != "layers" else [{kk: vv.to(DEV) for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
     model = sfs.Model(shape, wd)
     cfg = F.ModelConfig(**shape.asdict())
@@ -101,7 +101,7 @@ def test_forward_logits_at_widths_that_fill_no_tile(dims):
     sequence of 72 or 200 tokens: ragged tiles in every projection (rows, columns and the K of the down projection), ragged
     key tiles, and a vocabulary that ends inside a column tile."""
     shape = W.Shape(n_layers=2, mask_id=dims["vocab"] - 1, rms_eps=1e-5, rope_theta=10000.0, logit_scale=8.0, **dims)
-    w = W.model_weights(shape, seed=5)
+    w = W.model_weights(shape, seed=5, gain_std=0.2)
     wd = {k: (v.to(DEV) if k != "layers" else [{kk: vv.to(DEV) for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
     model = sfs.Model(shape, wd)
     cfg = F.ModelConfig(**shape.asdict())

@@ -14,7 +14,7 @@ from paper_2506_10848_b200 import workloads as W
 SHAPE = W.Shape(n_layers=3, d_model=64, n_heads=2, head_dim=32, d_ff=96, vocab=128, mask_id=127,
                 rms_eps=1e-5, rope_theta=10000.0, logit_scale=2.0)
 CFG = F.ModelConfig(**SHAPE.asdict())
-WTS = W.weights_to_numpy(W.model_weights(SHAPE, seed=5, std=0.2), np.float64)
+WTS = W.weights_to_numpy(W.model_weights(SHAPE, seed=5, std=0.2, gain_std=0.3), np.float64)   # every norm its own gains
 P, L = 6, 10
 S = P + L
 
