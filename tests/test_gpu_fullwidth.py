@@ -36,7 +36,7 @@ NOISE_MARGIN = 1.10                   # GPU-to-oracle distance over the distance
 @pytest.fixture(scope="module")
 def model2():
     shape = W.with_layers(W.LLADA_8B, 2)
-    w = W.model_weights(shape, seed=2, device=DEV, gain_std=0.2)      # every norm its own gains
+    w = W.model_weights(shape, seed=2, device=DEV)
     model = sfs.Model(shape, w)
     w_cpu = {k: (v.cpu() if k != "layers" else [{kk: vv.cpu() for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
     w32 = W.weights_to_numpy(w_cpu, np.float32)
