@@ -107,3 +107,26 @@ def test_cached_generation_schedule_span_and_restart():
     assert saw_fast
     y2, trace2 = G.generate_cached(cfg, w, prompt, L, SlowFastParams(), kp, kr, rho)
     assert y2 == y and [r.key() for r in trace2] == [r.key() for r in trace]
+
+
+def test_cached_generation_hands_the_span_of_an_accelerated_step_to_the_cache(monkeypatch):
+    """What the cache is told per step: the span [s_cycle, hi) when the step is an accelerated one, nothing otherwise
+    (the spans of the run above can cover the whole response, where the restriction is invisible in the sets)."""
+    dct = W.TINY.asdict(); dct["logit_scale"] = 60.0
+    shape = W.Shape(**dct)
+    cfg = F.ModelConfig(**shape.asdict())
+    w = W.weights_to_numpy(W.model_weights(shape, seed=0), np.float64)
+    prompt = W.prompt_ids(1, 32, 4094, seed=0)[0].tolist()
+    seen = []
+    real = G.C.cached_forward
+
+    def spy(*a, **k):
+        seen.append((k.get("span"), list(k.get("rows"))))
+        return real(*a, **k)
+
+    monkeypatch.setattr(G.C, "cached_forward", spy)
+    y, trace = G.generate_cached(cfg, w, prompt, 32, SlowFastParams(), 100, 4, 0.25)
+    assert len(seen) == len(trace) and any(r.phase == 1 for r in trace)
+    for r, (span, rows) in zip(trace, seen):
+        assert span == ((r.s, r.hi) if r.phase == 1 else None), (r.step, span)
+        assert all(32 <= q < 64 for q in rows)                        # logits rows are sequence positions of the response

@@ -89,6 +89,14 @@ def test_thresholds_are_strict_and_canonical():
     import struct
     tau32 = struct.unpack("f", struct.pack("f", 0.1))[0]
     assert exceeds(10 * one, 0.1) == (float(10 * one) * tau32 < float(one))
+    # around c = 0.1 the two readings part: float32(0.1) = 0.1 + 1.49e-9 moves the boundary by 40 units of S_q
+    from fractions import Fraction
+    flips = 0
+    for sq in range(10 * one - 60, 10 * one + 5):
+        want = Fraction(sq) * Fraction(tau32) < one               # exact rational arithmetic on the float the ABI carries
+        assert exceeds(sq, 0.1) == want, sq
+        flips += want != (Fraction(sq) * Fraction(1, 10) < one)
+    assert flips >= 30                                            # the window really separates the readings
 
 
 def test_top_k_ties_to_smaller_position():
