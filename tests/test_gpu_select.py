@@ -106,6 +106,8 @@ def test_lockstep_default_params(seed):
     (12, dict(max_steps=9, k_slow=1)),                       # the step budget runs out: forced last step
     (13, dict(tau_min_conf=-1.0, tau_high_conf=2.0, sigma2_stable=float("inf"), k_max=1, w_hist=1)),
     (14, dict(w_hist=8, k_max=12, sigma2_stable=400.0)),
+    (15, dict(k_max=3, w_hist=2, sigma2_stable=0.0)),        # no variance is below 0: every cycle ends by the K_max fallback
+    (16, dict(k_max=2, w_hist=5)),                           # the history cannot fill before K_max
 ])
 def test_lockstep_other_params(seed, pkw):
     run_lockstep(B=2, P=3, L=40, V=256, pkw=pkw, seed=seed)
@@ -282,6 +284,52 @@ def test_full_vocabulary_steps_where_the_cheap_pass_cannot_decide(case):
             n = int(sel_count[0])
             assert sel_pos[0, :n].tolist() == rec.positions and sel_tok[0, :n].tolist() == rec.tokens, (case, phase)
             assert trace[0].tolist()[:6] == [rec.phase, rec.s, rec.hi, rec.e_cand, rec.stable, len(rec.positions)], (case, phase)
+        sfs.sfs_check_device_status()
+    finally:
+        sfs.sfs_session_destroy(session)
+
+
+@pytest.mark.parametrize("V", [512, 126464])
+def test_thresholds_are_strict_where_the_confidence_equals_them(V):
+    """Rows with n equal maxima and nothing else within reach have S_q = n 2^28 exactly, i.e. c = 1/n.  With tau_min = 1/4
+    and tau_high = 1/2 (both exact in float32) the rows at c = 1/4 and c = 1/2 sit on the thresholds: the comparisons are
+    strict, on short rows (one-pass statistics) and on full-vocabulary rows (the cheap pass cannot decide them)."""
+    L, P, B = 16, 0, 1
+    n_max = [1, 2, 3, 4, 5, 2, 4, 1, 3, 4, 2, 6, 4, 2, 1, 4]
+    logits = torch.full((L, V), -200.0, dtype=torch.float32)
+    g = torch.Generator().manual_seed(V)
+    for i, n in enumerate(n_max):
+        logits[i, torch.randperm(V, generator=g)[:n]] = 1.5
+    logits = logits.to(torch.bfloat16)
+    stats = RS.row_stats(W.bf16_bits(logits))
+    assert [int(s) for s in stats["sq"]] == [n << 28 for n in n_max]
+    po, pg = params_pair(tau_min_conf=0.25, tau_high_conf=0.5)
+    session = sfs.sfs_select_session_create(V, B, L)
+    try:
+        for phase, span in ((SLOW, None), (FAST, (1, 15))):
+            tokens = torch.full((B, L), V - 1, dtype=torch.int32, device=DEV)
+            mask = torch.ones((B, L), dtype=torch.uint8, device=DEV)
+            state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+            sfs.sfs_state_init(state, B, L, pg)
+            ost = SlowFastState.fresh(L, po)
+            if phase == FAST:
+                write_state(state, 0, phase=1, s_cycle=span[0], hi=span[1])
+                ost.phase, ost.s_cycle, ost.hi = FAST, span[0], span[1]
+            rows = torch.arange(L, dtype=torch.int32, device=DEV)
+            sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+            sel_pos = torch.zeros((B, L), dtype=torch.int32, device=DEV); sel_tok = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+            trace = torch.zeros((B, sfs.TRACE_INTS), dtype=torch.int32, device=DEV)
+            sfs.sfs_select(session, logits.to(DEV), sfs.LOGITS_BF16, V, rows, None, L, tokens, mask, B, L, P, state, pg,
+                           sel_count, sel_pos, sel_tok, trace=trace)
+            torch.cuda.synchronize()
+            rec = slowfast_step(ost, {i: int(stats["argmax"][i]) for i in range(L)}, {i: int(stats["sq"][i]) for i in range(L)}, po)
+            n = int(sel_count[0])
+            assert sel_pos[0, :n].tolist() == rec.positions and sel_tok[0, :n].tolist() == rec.tokens, phase
+            assert trace[0].tolist()[:6] == [rec.phase, rec.s, rec.hi, rec.e_cand, rec.stable, len(rec.positions)], phase
+            if phase == SLOW:
+                assert rec.e_cand == 14                           # position 15 (c = 1/4) does not reach tau_min, 14 (c = 1) does
+            else:
+                assert rec.positions == [7, 14]                   # c = 1 only: the rows at c = 1/2 stay masked
         sfs.sfs_check_device_status()
     finally:
         sfs.sfs_session_destroy(session)
