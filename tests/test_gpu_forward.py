@@ -94,6 +94,44 @@ def test_forward_logits_tiny_within_tolerance():
         model.close()
 
 
+def test_forward_logits_with_peaked_attention():
+    """Random-init projections give nearly uniform attention, where an error in the rotary embedding or in the score scale
+    moves the logits only at second order.  Here W_q and W_k are eight times larger: the softmax is peaked, positions matter
+    at first order, and so does the rounding of q and k — the bar is the distance of the rounding-only model of a bf16
+    pipeline from the same oracle, plus 15 %."""
+    shape = W.TINY
+    w = W.model_weights(shape, seed=8, gain_std=0.2)
+    for lw in w["layers"]:
+        lw["wq"] = (lw["wq"].float() * 8.0).to(torch.bfloat16)
+        lw["wk"] = (lw["wk"].float() * 8.0).to(torch.bfloat16)
+    wd = {k: (v.to(DEV) if k != "layers" else [{kk: vv.to(DEV) for kk, vv in lw.items()} for lw in v]) for k, v in w.items()}
+    model = sfs.Model(shape, wd)
+    cfg = F.ModelConfig(**shape.asdict())
+    w64 = W.weights_to_numpy(w, np.float64)
+    B, P, L = 2, 40, 160
+    S = P + L
+    tok = torch.cat([W.prompt_ids(B, P, 4094, seed=3), torch.full((B, L), shape.mask_id, dtype=torch.int32)], dim=1)
+    tok[:, P + 5:P + 60:3] = W.prompt_ids(B, 19, 4094, seed=4)        # a partly decoded response: rows differ by more than position
+    session = sfs.sfs_session_create(model, B, S)
+    try:
+        rows = [(b, t) for b in range(B) for t in range(0, S, 7)]
+        d_rows = torch.tensor([b * S + t for (b, t) in rows], dtype=torch.int32, device=DEV)
+        lg = torch.zeros((len(rows), shape.vocab), dtype=torch.float32, device=DEV)
+        sfs.sfs_forward(session, tok.to(DEV), B, S, d_rows, None, len(rows), lg, sfs.LOGITS_F32)
+        sfs.sfs_check_device_status()
+        ref = F.forward(cfg, w64, tok.numpy(), rows=rows, dtype=np.float64)
+        got = lg.cpu().double().numpy()
+        emu = np.concatenate([forward_bf16_points(cfg, w, tok[b].numpy(), [t for (bb, t) in rows if bb == b]) for b in range(B)])
+        rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+        rel_model = np.linalg.norm(emu - ref) / np.linalg.norm(ref)
+        print(f"peaked attention: GPU vs oracle rel_l2={rel:.4g}, rounding-only model vs oracle {rel_model:.4g}")
+        assert rel <= 1.15 * rel_model and rel <= 3e-2, (rel, rel_model)
+        assert np.abs(got - ref).max() <= 1.4 * np.abs(emu - ref).max()
+    finally:
+        sfs.sfs_session_destroy(session)
+        model.close()
+
+
 @pytest.mark.parametrize("dims", [dict(d_model=384, n_heads=3, head_dim=128, d_ff=1000, vocab=5000),
                                   dict(d_model=640, n_heads=10, head_dim=64, d_ff=1736, vocab=8200)])
 def test_forward_logits_at_widths_that_fill_no_tile(dims):

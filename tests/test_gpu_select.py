@@ -333,3 +333,40 @@ def test_thresholds_are_strict_where_the_confidence_equals_them(V):
         sfs.sfs_check_device_status()
     finally:
         sfs.sfs_session_destroy(session)
+
+
+@pytest.mark.parametrize("min_high,expect", [(2, [3, 9]), (3, [3])])
+def test_fast_step_with_exactly_the_minimum_number_of_confident_rows(min_high, expect):
+    """An accelerated step whose span holds exactly two rows above tau_high: with a minimum of two the confident set is
+    taken as it is, with a minimum of three the step falls back to the k_fast most confident rows (here one: of the two
+    rows at c = 1 the one at the smaller position)."""
+    V, L, P, B = 512, 16, 0, 1
+    logits = torch.full((L, V), -200.0, dtype=torch.float32)
+    g = torch.Generator().manual_seed(7)
+    for i in range(L):
+        logits[i, torch.randperm(V, generator=g)[: (1 if i in (3, 9) else 3)]] = 0.5      # c = 1 at rows 3 and 9, 1/3 elsewhere
+    logits = logits.to(torch.bfloat16)
+    stats = RS.row_stats(W.bf16_bits(logits))
+    po, pg = params_pair(tau_high_conf=0.5, min_high_count=min_high, k_fast=1)
+    session = sfs.sfs_select_session_create(V, B, L)
+    try:
+        tokens = torch.full((B, L), V - 1, dtype=torch.int32, device=DEV)
+        mask = torch.ones((B, L), dtype=torch.uint8, device=DEV)
+        state = torch.zeros((B, sfs.STATE_INTS), dtype=torch.int32, device=DEV)
+        sfs.sfs_state_init(state, B, L, pg)
+        write_state(state, 0, phase=1, s_cycle=0, hi=L)
+        ost = SlowFastState.fresh(L, po)
+        ost.phase, ost.s_cycle, ost.hi = FAST, 0, L
+        rows = torch.arange(L, dtype=torch.int32, device=DEV)
+        sel_count = torch.zeros(B, dtype=torch.int32, device=DEV)
+        sel_pos = torch.zeros((B, L), dtype=torch.int32, device=DEV); sel_tok = torch.zeros((B, L), dtype=torch.int32, device=DEV)
+        sfs.sfs_select(session, logits.to(DEV), sfs.LOGITS_BF16, V, rows, None, L, tokens, mask, B, L, P, state, pg,
+                       sel_count, sel_pos, sel_tok)
+        torch.cuda.synchronize()
+        sfs.sfs_check_device_status()
+        rec = slowfast_step(ost, {i: int(stats["argmax"][i]) for i in range(L)}, {i: int(stats["sq"][i]) for i in range(L)}, po)
+        n = int(sel_count[0])
+        assert sel_pos[0, :n].tolist() == rec.positions == expect
+        assert sel_tok[0, :n].tolist() == rec.tokens
+    finally:
+        sfs.sfs_session_destroy(session)
